@@ -336,12 +336,16 @@ def test_batch_rollout_equals_frame_by_frame():
 
 
 def test_opponent_box_y_edges_are_half_open():
-    # opponent held by the clamp at opy = 0 (ball centre above its centre)
-    e = env(bx=3500, vx=-600, by=4096, vy=0, opy=0); e.frame(0); assert e.vx == -600
-    e = env(bx=3500, vx=-600, by=4095, vy=0, opy=0); e.frame(0); assert e.vx == 616
-    # held at the bottom clamp, ball just above the paddle's top edge
-    e = env(bx=3500, vx=-600, by=45056 - 512, vy=0, opy=45056); e.frame(0); assert e.vx == -600
-    e = env(bx=3500, vx=-600, by=45056 - 511, vy=0, opy=45056); e.frame(0); assert e.vx == 616
+    # the opponent first tracks by 512 (0 -> 512); box is [512, 4608)
+    e = env(bx=3500, vx=-600, by=4608, vy=0, opy=0); e.frame(0)
+    assert (e.opy, e.vx) == (512, -600)
+    e = env(bx=3500, vx=-600, by=4607, vy=0, opy=0); e.frame(0)
+    assert (e.opy, e.vx) == (512, 616)
+    # tracking upwards 45056 -> 44544; the ball's bottom edge must pass 44544
+    e = env(bx=3500, vx=-600, by=44544 - 512, vy=0, opy=45056); e.frame(0)
+    assert (e.opy, e.vx) == (44544, -600)
+    e = env(bx=3500, vx=-600, by=44544 - 511, vy=0, opy=45056); e.frame(0)
+    assert (e.opy, e.vx) == (44544, 616)
 
 
 def test_respawn_point_key_counts_both_scores():
