@@ -1,0 +1,36 @@
+// Launch interface between the C ABI (pong_api.cu) and the kernels
+// (pong_kernels.cu).  Plain pointers and sizes only.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "pong_rules.cuh"
+
+namespace pong {
+
+struct LaunchArgs {
+    int4 *plane0;              // [n] {bx, by, vx, vy}
+    int4 *plane1;              // [n] {apy, opy, packed counters, episode}
+    long long *stats;          // [3] episodes, sum of returns, sum of lengths
+    const uint8_t *actions;    // explicit mode: [T][n] action bytes
+    float *obs;                // vector mode: [T][n][6]
+    uint8_t *ring;             // pixel mode: [n][4][84][84]
+    float *reward;             // [T][n]
+    uint8_t *done;             // [T][n]
+    RoundKeys rk;              // Philox round keys of the seed
+    unsigned long long t0;     // global agent step of the first step
+    uint32_t env_id_base;
+    int n;
+    int T;
+    int action_mode;           // 0 Philox, 1 sticky, 2 explicit, 3 constant
+    int const_action;          // mode 3
+    int frameskip;
+};
+
+// Each returns the cudaError_t of the launch (cudaGetLastError).
+cudaError_t launch_reset(const LaunchArgs &a, cudaStream_t s);          // state + optional obs / ring
+cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s);
+cudaError_t launch_rollout_pixels(const LaunchArgs &a, int sm_count, cudaStream_t s);
+cudaError_t launch_fill_actions(const LaunchArgs &a, int sticky, uint8_t *out, cudaStream_t s);
+
+}  // namespace pong

@@ -1,0 +1,65 @@
+"""The C-ABI library builds, loads and exports every symbol the header
+declares (no compute calls: this runs without a GPU)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2603_12145_b200 import build, pong
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "pong.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(pong_[a-z_]+)\s*\(", text)))
+
+
+def test_library_builds_and_exports_every_declared_symbol():
+    path = build.build()
+    lib = ctypes.CDLL(path)
+    names = declared_symbols()
+    assert len(names) >= 15
+    for name in names:
+        assert hasattr(lib, name), name
+    assert set(names) == set(pong.EXPORTS)
+
+
+def test_strerror_and_null_handles_without_gpu():
+    L = pong.load(build_if_missing=True)
+    assert pong.strerror(0) == "ok"
+    for code in range(-6, 0):
+        assert pong.strerror(code) != "unknown error code"
+    assert pong.strerror(-99) == "unknown error code"
+    # NULL handle / NULL out-pointer are rejected before any CUDA call
+    assert L.pong_reset(None, None) == -2
+    assert L.pong_step(None, None, None, None, None) == -2
+    assert L.pong_rollout(None, 1, 0, None, None, None, None) == -2
+    assert L.pong_fill_actions(None, 1, 0, None) == -2
+    assert L.pong_episode_stats(None, None, None, None, 0) == -2
+    assert L.pong_get_state(None, None, None) == -2
+    assert L.pong_set_state(None, None, 0) == -2
+    assert L.pong_set_stream(None, None) == -2
+    assert L.pong_destroy(None) == 0
+    assert L.pong_create(None, 4, 0) == -2
+    h = ctypes.c_void_p()
+    assert L.pong_create(ctypes.byref(h), 0, 0) == -1
+    cfg = pong._Config(2, 1, 0)
+    assert L.pong_create_ex(ctypes.byref(h), 4, 0, ctypes.byref(cfg)) == -1
+    cfg = pong._Config(0, 17, 0)
+    assert L.pong_create_ex(ctypes.byref(h), 4, 0, ctypes.byref(cfg)) == -1
+    cfg = pong._Config(0, 1, -1)
+    assert L.pong_create_ex(ctypes.byref(h), 4, 0, ctypes.byref(cfg)) == -1
+
+
+def test_no_cpu_fallback_without_device():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present")
+    with pytest.raises((pong.PongError, RuntimeError)):
+        pong.PongEnv(4, 0)
+    with pytest.raises(pong.PongError) as ei:
+        pong.pong_create(4, 0)
+    assert ei.value.code == -4
