@@ -1,0 +1,327 @@
+#!/usr/bin/env python
+"""Benchmark of the batched Pong rollout: env-steps/s on B200 and the achieved
+fraction of the HBM roofline.
+
+One "step" of this benchmark is one fused rollout launch over the whole batch:
+N = 65,536 envs x T = 128 agent steps with in-kernel Philox actions, vector
+observations float32[T,N,6] plus reward and done buffers, and the episode
+statistics reduction, i.e. 8,388,608 env-steps and 243 MB written per step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints one JSON line (rank 0).  With --gpus N > 1 it must be launched with
+torchrun, one rank per GPU; each rank simulates its own 65,536 envs (global env
+ids rank*65536 ...), so the scaling is weak and there is no data-path
+collective.  --impl reference times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+N_ENVS = 65536
+T_STEPS = 128
+SEED = 0
+METRIC = "env-steps/sec on 1 B200 and achieved HBM GB/s fraction of roofline"
+UNIT = "env-steps/s"
+WORKLOAD = "fused vector-obs rollout, N=65536 envs, T=128 steps per launch, in-kernel Philox actions"
+# Algorithmic bytes per env-step: obs 24 + reward 4 + done 1 written, plus the
+# 32-byte state read and written once per launch (64 / T).
+BYTES_PER_ENV_STEP = 29.0 + 64.0 / T_STEPS
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the rollout
+# kernel from an ncu capture of this workload (see profiles/); None when the
+# kernel has changed since the counters were taken.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML (read-only)."""
+
+    def __init__(self, index, period=0.01):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples = []          # (time, sm_mhz, reasons bitmask)
+        self.max_mhz = None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._halt.is_set():
+            try:
+                mhz = int(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM))
+                try:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev))
+                except Exception:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev))
+                self.samples.append((time.perf_counter(), mhz, reasons))
+            except Exception:
+                pass
+            self._halt.wait(self.period)
+
+    def stop(self):
+        self._halt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+
+    def summary(self, t0, t1):
+        names = {0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+                 0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+                 0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+        inside = [s for s in self.samples if t0 <= s[0] <= t1]
+        where = "timed region"
+        if not inside:
+            inside, where = self.samples, "whole run (timed region shorter than the sampling period)"
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0,
+                    "note": "NVML unavailable"}
+        mhz = sorted(s[1] for s in inside)
+        mask = 0
+        for s in inside:
+            mask |= s[2]
+        reasons = [n for b, n in names.items() if mask & b]
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz, "reasons": reasons,
+                "samples": len(inside), "sampled_over": where}
+
+
+def physical_gpu_index(local):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local])
+        except Exception:
+            return local
+    return local
+
+
+def cpu_oracle_rate(budget_s, n_sample=8192, min_reps=1):
+    """Env-steps/s of the CPU oracle, as it stands, on one host thread: envs
+    0..n_sample-1 of the same workload, T=128 steps per call, repeated until the
+    time budget is used."""
+    import oracle
+    o = oracle.OraclePong(n_sample, SEED)
+    o.rollout(T_STEPS, 0)                       # warm-up (page-in, first touch)
+    steps, reps, t0 = 0, 0, time.perf_counter()
+    while True:
+        o.rollout(T_STEPS, 0)
+        steps += n_sample * T_STEPS
+        reps += 1
+        dt = time.perf_counter() - t0
+        if reps >= min_reps and dt >= budget_s:
+            break
+    return steps / dt, reps, dt
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    n_sample = 8192
+    import oracle
+    o = oracle.OraclePong(n_sample, SEED)
+    for _ in range(max(args.warmup, 1)):
+        o.rollout(T_STEPS, 0)
+    # each step: T=128 oracle steps of the first 8192 envs of the workload;
+    # cap the run at about two minutes whatever --steps says
+    k = max(1, min(args.steps, 200))
+    t0 = time.perf_counter()
+    done_steps = 0
+    for i in range(k):
+        o.rollout(T_STEPS, 0)
+        done_steps += 1
+        if time.perf_counter() - t0 > 120.0:
+            break
+    dt = time.perf_counter() - t0
+    value = done_steps * n_sample * T_STEPS / dt
+    sample = "envs 0..%d of the workload, T=%d per step, %d steps, single thread" % (
+        n_sample - 1, T_STEPS, done_steps)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": done_steps, "warmup": max(args.warmup, 1), "ms_per_step": dt / done_steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
+        "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=8)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2603_12145_b200 import pong
+    from paper_2603_12145_b200.inputs import explicit_actions
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if world != args.gpus:
+        raise SystemExit("--gpus %d needs torchrun with %d ranks (WORLD_SIZE=%d)" % (
+            args.gpus, args.gpus, world))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pong.load()
+    warmup = max(args.warmup, 3)
+    steps = max(args.steps, 1)
+
+    env = pong.PongEnv(N_ENVS, SEED, env_id_base=rank * N_ENVS)
+    obs = torch.empty((T_STEPS, N_ENVS, 6), dtype=torch.float32, device="cuda")
+    reward = torch.empty((T_STEPS, N_ENVS), dtype=torch.float32, device="cuda")
+    done = torch.empty((T_STEPS, N_ENVS), dtype=torch.uint8, device="cuda")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    for _ in range(warmup):
+        env.rollout(T_STEPS, pong.ACT_PHILOX, None, obs, reward, done)
+    barrier()
+
+    # ---- device-resident timing: K launches, CUDA events on the launching stream
+    n_seg = 5 if steps >= 50 else 1
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_seg + 1)]
+    launches0 = env.launches
+    w0 = time.perf_counter()
+    marks[0].record()
+    for s in range(n_seg):
+        lo, hi = steps * s // n_seg, steps * (s + 1) // n_seg
+        for _ in range(hi - lo):
+            env.rollout(T_STEPS, pong.ACT_PHILOX, None, obs, reward, done)
+        marks[s + 1].record()
+    torch.cuda.synchronize()
+    w1 = time.perf_counter()
+    launches = env.launches - launches0
+    barrier()
+    ms_total = marks[0].elapsed_time(marks[-1])
+    seg_rates = []
+    for s in range(n_seg):
+        k = steps * (s + 1) // n_seg - steps * s // n_seg
+        seg_rates.append(k * N_ENVS * T_STEPS / (marks[s].elapsed_time(marks[s + 1]) * 1e-3))
+    if world > 1:
+        tmax = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms_total = float(tmax.item())
+    stats = env.episode_stats()
+
+    # ---- end to end: host buffers in, host buffers out, through pong_rollout_host
+    e2e_steps = max(args.e2e_steps, 1)
+    acts_h = torch.from_numpy(explicit_actions(T_STEPS, N_ENVS, seed=SEED)).pin_memory()
+    obs_h = torch.empty((T_STEPS, N_ENVS, 6), dtype=torch.float32).pin_memory()
+    rew_h = torch.empty((T_STEPS, N_ENVS), dtype=torch.float32).pin_memory()
+    done_h = torch.empty((T_STEPS, N_ENVS), dtype=torch.uint8).pin_memory()
+    env._stream()
+    for _ in range(2):
+        pong.pong_rollout_host(env.h, T_STEPS, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
+    barrier()
+    e0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        pong.pong_rollout_host(env.h, T_STEPS, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - e0
+    if world > 1:
+        tmax = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_s = float(tmax.item())
+    sampler.stop()
+    barrier()
+
+    env_steps_per_launch = N_ENVS * T_STEPS
+    value = world * steps * env_steps_per_launch / (ms_total * 1e-3)
+    peak, peak_kind = measured_peak()
+    kernel_ms = ms_total / steps
+    achieved = env_steps_per_launch * BYTES_PER_ENV_STEP / (kernel_ms * 1e-3) / 1e9
+    h2d = acts_h.numel()
+    d2h = obs_h.numel() * 4 + rew_h.numel() * 4 + done_h.numel()
+
+    if rank == 0:
+        mean = sum(seg_rates) / len(seg_rates)
+        std = (sum((x - mean) ** 2 for x in seg_rates) / len(seg_rates)) ** 0.5
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": warmup, "ms_per_step": kernel_ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "config": {
+                "workload": WORKLOAD, "n_envs_per_gpu": N_ENVS, "T": T_STEPS, "seed": SEED,
+                "env_steps_per_step": env_steps_per_launch,
+                "l2": "each step writes 243 MB of outputs, larger than the 126 MB L2; no flush",
+                "parallelism": "env shards per GPU, no collective" if world > 1 else "single GPU",
+            },
+            "roofline": {
+                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "algorithmic_bytes_per_launch": env_steps_per_launch * BYTES_PER_ENV_STEP,
+                "bytes_per_env_step": BYTES_PER_ENV_STEP,
+                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "kernel": "k_rollout_vector", "kernel_ms": kernel_ms,
+            },
+            "e2e": {"value": world * e2e_steps * env_steps_per_launch / e2e_s, "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+                    "api": "pong_rollout_host, pinned host buffers, explicit actions"},
+            "gpu_launches": int(launches),
+            "clocks": sampler.summary(w0, w1),
+            "segments": {"n": n_seg, "mean": mean, "std": std, "cv": std / mean},
+            "episode_stats": {"episodes": stats[0], "sum_return": stats[1], "sum_length": stats[2]},
+        }
+        if world == 1:
+            rate, reps, dt = cpu_oracle_rate(args.cpu_seconds)
+            line["cpu_baseline"] = {
+                "value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
+                "host_cores": os.cpu_count(),
+                "sample": "envs 0..8191 of the workload, T=128 per call, %d calls, %.1f s, "
+                          "single thread" % (reps, dt)}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
