@@ -301,7 +301,7 @@ def main():
                 "algorithmic_bytes_per_launch": env_steps_per_launch * BYTES_PER_ENV_STEP,
                 "bytes_per_env_step": BYTES_PER_ENV_STEP,
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "kernel": "k_rollout_vector", "kernel_ms": kernel_ms,
+                "kernel": "k_rollout_vector_tma", "kernel_ms": kernel_ms,
             },
             "e2e": {"value": world * e2e_steps * env_steps_per_launch / e2e_s, "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,

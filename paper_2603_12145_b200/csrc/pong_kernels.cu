@@ -3,7 +3,13 @@
 //   k_reset            state planes <- reset(seed, env, 0); optional initial obs
 //   k_reset_pixels     reset frame into all four ring slots
 //   k_rollout_vector   one thread per env, state in registers across T steps,
-//                      streams obs / reward / done to HBM
+//                      streams obs / reward / done to HBM with per-thread stores
+//                      (any n, T, frameskip and action mode)
+//   k_rollout_vector_tma  the same rollout for the common case (Philox actions,
+//                      frameskip 1, aligned n / t / T): outputs are staged in shared
+//                      memory 8 steps at a time and leave through TMA tensor stores,
+//                      the Philox block of the next four steps is interleaved with
+//                      the physics of the current four, rare paths are warp-uniform
 //   k_rollout_pixels   one thread per env for the physics, one warp per frame
 //                      for the rasteriser; frames are staged in shared memory
 //                      and leave through bulk async copies (16-byte granules)
@@ -11,6 +17,8 @@
 //
 // No kernel waits on another block, on a flag or on an mbarrier; the only
 // blocking instructions are __syncthreads and cp.async.bulk.wait_group.
+#include <cuda.h>
+
 #include "pong_kernels.cuh"
 
 namespace pong {
@@ -38,6 +46,53 @@ __device__ __forceinline__ int pick_action(uint32_t word, const Env &e, const ui
     if (MODE == 1) return sticky_repeat(word) ? e.prev : uniform_action(word);
     if (MODE == 2) return decode_action_byte(*act, e.prev);
     return const_action;
+}
+
+// ---- asynchronous copy helpers ---------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+// Bulk async copy of `bytes` (multiple of 16) from shared to global memory;
+// both addresses 16-byte aligned.
+__device__ __forceinline__ void bulk_store(void *gdst, const void *ssrc, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 :: "l"(gdst), "r"(smem_addr(ssrc)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit()
+{
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int PENDING>
+__device__ __forceinline__ void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(PENDING) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem()
+{
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// TMA tensor store of a 2-D box from shared memory; (x, y) is the box origin in
+// elements of the tensor map, x * element size a multiple of 16 bytes.  Parts of
+// the box outside the tensor are not written.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, const void *ssrc, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 :: "l"(map), "r"(smem_addr(ssrc)), "r"(x), "r"(y) : "memory");
+}
+// Programmatic dependent launch: wait for the preceding kernel of the stream to
+// complete and flush / let the following kernel start its prologue.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+__device__ __forceinline__ void grid_dependency_launch()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
 // ---- reset --------------------------------------------------------------------------
@@ -128,8 +183,181 @@ static void launch_vec_mode(const LaunchArgs &a, bool full, cudaStream_t s)
         launch_vec_full<MODE, 0>(a, full, s);
 }
 
+// ---- vector rollout, TMA path ---------------------------------------------------------
+
+constexpr int kTmaBlock = 64;  // envs per block (two warps)
+constexpr int kTmaStage = 8;   // agent steps staged in shared memory per TMA store
+
+struct VectorMaps {
+    CUtensorMap obs;     // [T][3n] 8-byte elements (pairs of floats), box 3*kTmaBlock x kTmaStage
+    CUtensorMap reward;  // [T][n] float32, box kTmaBlock x kTmaStage
+    CUtensorMap done;    // [T][n] uint8, box kTmaBlock x kTmaStage
+};
+
+// Requirements (checked by the launcher): frameskip 1, t0 % 4 == 0,
+// T % kTmaStage == 0, n % 16 == 0 (row pitches are multiples of 16 bytes).
+// Threads past n run a copy of env n-1 so that every warp stays whole; their
+// outputs fall outside the tensor maps and are dropped by the TMA unit.
+template <int MODE>
+__global__ void __launch_bounds__(kTmaBlock) k_rollout_vector_tma(const __grid_constant__ LaunchArgs a,
+                                                                  const __grid_constant__ VectorMaps maps)
+{
+    __shared__ __align__(128) float s_obs[2][kTmaStage][kTmaBlock * 6];
+    __shared__ __align__(128) float s_reward[2][kTmaStage][kTmaBlock];
+    __shared__ __align__(128) uint8_t s_done[2][kTmaStage][kTmaBlock];
+
+    const int tid = threadIdx.x;
+    const int n0 = blockIdx.x * kTmaBlock;
+    const bool valid = n0 + tid < a.n;
+    const int n = valid ? n0 + tid : a.n - 1;
+    const uint32_t env_id = a.env_id_base + (uint32_t)n;
+    Tally tally = {0, 0, 0};
+
+    // Philox block of the first four steps: independent of the state, so it runs
+    // before the wait on the previous kernel.
+    unsigned long long g = a.t0 >> 2;
+    PhiloxPipe pipe;
+    philox_start(pipe, g, env_id);
+    philox_rounds<0, 10>(pipe, a.rk);
+
+    grid_dependency_wait();
+    FastEnv e;
+    {
+        Env q;
+        load_env(q, a.plane0, a.plane1, n);
+        to_fast(e, q);
+    }
+    grid_dependency_launch();
+
+    int buf = 0;
+    for (int t = 0; t < a.T; t += kTmaStage) {
+        // the store that last read this buffer is the older of the two in flight
+        if (tid == 0) bulk_wait_read<1>();
+        __syncthreads();
+#pragma unroll
+        for (int q = 0; q < kTmaStage / 4; ++q) {
+            const uint32_t w[4] = {pipe.c0, pipe.c1, pipe.c2, pipe.c3};
+            ++g;
+            philox_start(pipe, g, env_id);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (j == 0) philox_rounds<0, 3>(pipe, a.rk);
+                if (j == 1) philox_rounds<3, 6>(pipe, a.rk);
+                if (j == 2) philox_rounds<6, 8>(pipe, a.rk);
+                if (j == 3) philox_rounds<8, 10>(pipe, a.rk);
+                const int s = q * 4 + j;
+                int action = uniform_action(w[j]);
+                if (MODE == 1) action = sticky_repeat(w[j]) ? e.prev : action;
+                e.prev = action;
+                float r;
+                int dn;
+                fast_frame(e, action, env_id, a.rk, tally, r, dn);
+                float2 *o = reinterpret_cast<float2 *>(&s_obs[buf][s][tid * 6]);
+                o[0] = make_float2(scale_obs(e.bx), scale_obs(e.by));
+                o[1] = make_float2(scale_obs(e.vx), scale_obs(e.vy));
+                o[2] = make_float2(scale_obs(e.apy), scale_obs(e.opy));
+                s_reward[buf][s][tid] = r;
+                s_done[buf][s][tid] = (uint8_t)dn;
+            }
+        }
+        fence_async_smem();
+        __syncthreads();
+        if (tid == 0) {
+            tma_store_2d(&maps.obs, &s_obs[buf][0][0], n0 * 3, t);
+            tma_store_2d(&maps.reward, &s_reward[buf][0][0], n0, t);
+            tma_store_2d(&maps.done, &s_done[buf][0][0], n0, t);
+            bulk_commit();
+        }
+        buf ^= 1;
+    }
+    if (valid) {
+        Env q;
+        from_fast(q, e);
+        store_env(q, a.plane0, a.plane1, n);
+    } else {
+        tally.episodes = 0;
+        tally.sum_return = 0;
+        tally.sum_length = 0;
+    }
+    flush_tally(tally, a.stats);
+    if (tid == 0) bulk_wait_read<0>();
+}
+
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                      const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                      const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up once through the runtime (no link
+// against libcuda); nullptr if this driver does not have it.
+static TensorMapEncodeFn tensor_map_encoder()
+{
+    static TensorMapEncodeFn fn = []() -> TensorMapEncodeFn {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        return reinterpret_cast<TensorMapEncodeFn>(p);
+    }();
+    return fn;
+}
+
+static bool encode_rows(TensorMapEncodeFn enc, CUtensorMap *m, CUtensorMapDataType type, void *base,
+                        uint64_t row_elems, uint64_t rows, uint64_t row_bytes, uint32_t box_elems,
+                        uint32_t box_rows)
+{
+    const cuuint64_t dims[2] = {row_elems, rows};
+    const cuuint64_t strides[1] = {row_bytes};
+    const cuuint32_t box[2] = {box_elems, box_rows};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    return enc(m, type, 2, base, dims, strides, box, elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Launches the TMA path if the call qualifies; returns false (nothing launched)
+// if it does not, so that the caller uses the general kernel.
+static bool try_launch_vector_tma(const LaunchArgs &a, cudaStream_t s, cudaError_t *err)
+{
+    if (a.action_mode > 1 || a.frameskip != 1) return false;
+    if (a.n % 16 != 0 || a.t0 % 4 != 0 || a.T % kTmaStage != 0) return false;
+    const uintptr_t bases = reinterpret_cast<uintptr_t>(a.obs) | reinterpret_cast<uintptr_t>(a.reward) |
+                            reinterpret_cast<uintptr_t>(a.done);
+    if (bases % 16 != 0) return false;  // tensor maps need 16-byte aligned bases
+    TensorMapEncodeFn enc = tensor_map_encoder();
+    if (enc == nullptr) return false;
+    VectorMaps maps;
+    const uint64_t n = (uint64_t)a.n, T = (uint64_t)a.T;
+    if (!encode_rows(enc, &maps.obs, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, a.obs, n * 3, T, n * 24,
+                     kTmaBlock * 3, kTmaStage) ||
+        !encode_rows(enc, &maps.reward, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.reward, n, T, n * 4,
+                     kTmaBlock, kTmaStage) ||
+        !encode_rows(enc, &maps.done, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.done, n, T, n, kTmaBlock,
+                     kTmaStage))
+        return false;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((a.n + kTmaBlock - 1) / kTmaBlock);
+    cfg.blockDim = dim3(kTmaBlock);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (a.action_mode == 0)
+        *err = cudaLaunchKernelEx(&cfg, k_rollout_vector_tma<0>, a, maps);
+    else
+        *err = cudaLaunchKernelEx(&cfg, k_rollout_vector_tma<1>, a, maps);
+    return true;
+}
+
 cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s)
 {
+    cudaError_t tma_err = cudaSuccess;
+    if (try_launch_vector_tma(a, s, &tma_err)) return tma_err != cudaSuccess ? tma_err : cudaGetLastError();
     const bool full = (a.t0 % 4 == 0) && (a.T % 4 == 0);
     switch (a.action_mode) {
     case 0: launch_vec_mode<0>(a, full, s); break;
@@ -146,32 +374,6 @@ constexpr int kPixThreads = 128;  // 4 warps; also the largest env count of a bl
 constexpr int kPixWarps = kPixThreads / 32;
 constexpr int kPixBufPerWarp = 3;  // staging frames per warp, used round-robin
 constexpr int kPixSmemBytes = kPixWarps * kPixBufPerWarp * kFrameBytes + kPixThreads * 4 + kPixThreads;
-
-__device__ __forceinline__ uint32_t smem_addr(const void *p)
-{
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-
-// Bulk async copy of `bytes` (multiple of 16) from shared to global memory;
-// both addresses 16-byte aligned.
-__device__ __forceinline__ void bulk_store(void *gdst, const void *ssrc, uint32_t bytes)
-{
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
-                 :: "l"(gdst), "r"(smem_addr(ssrc)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void bulk_commit()
-{
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-template <int PENDING>
-__device__ __forceinline__ void bulk_wait_read()
-{
-    asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(PENDING) : "memory");
-}
-__device__ __forceinline__ void fence_async_smem()
-{
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-}
 
 // One warp paints one 84x84 frame into shared memory.  Output pixel (i, j)
 // samples source row i*192/84 and source column j*160/84; the agent's paddle

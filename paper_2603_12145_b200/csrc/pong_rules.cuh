@@ -232,6 +232,123 @@ __device__ __forceinline__ int agent_step(Env &e, int action, int frameskip_rt,
     }
 }
 
+// ---- warp-uniform variant of the frame ------------------------------------------------
+// Same arithmetic as physics_frame, organised for a warp whose 32 lanes are all
+// live: the two rare paths (paddle bounce, score / episode end) sit behind
+// warp-uniform votes and commit their results per lane with selects, so the common
+// path is straight-line code.  The frame counter is kept as frames left in the
+// episode (kMaxFrames - len) so that the end test is a compare with zero.
+struct FastEnv {
+    int bx, by, vx, vy, apy, opy;
+    int sa, so, left, episode, prev;
+};
+
+__device__ __forceinline__ void to_fast(FastEnv &f, const Env &e)
+{
+    f.bx = e.bx; f.by = e.by; f.vx = e.vx; f.vy = e.vy; f.apy = e.apy; f.opy = e.opy;
+    f.sa = e.sa; f.so = e.so; f.left = kMaxFrames - e.len; f.episode = e.episode; f.prev = e.prev;
+}
+
+__device__ __forceinline__ void from_fast(Env &e, const FastEnv &f)
+{
+    e.bx = f.bx; e.by = f.by; e.vx = f.vx; e.vy = f.vy; e.apy = f.apy; e.opy = f.opy;
+    e.sa = f.sa; e.so = f.so; e.len = kMaxFrames - f.left; e.episode = f.episode; e.prev = f.prev;
+}
+
+// Score and / or episode end.  Run by the whole warp when any lane has an event;
+// only lanes with `ev` commit.  `out` says the ball left the court on this lane.
+__device__ __forceinline__ void fast_event(FastEnv &e, bool ev, bool out, uint32_t env_id,
+                                           const RoundKeys &rk, Tally &tally, float &reward,
+                                           int &done)
+{
+    const bool agent_point = e.bx > 0;
+    int sa = e.sa + ((out && agent_point) ? 1 : 0);
+    int so = e.so + ((out && !agent_point) ? 1 : 0);
+    const float r = out ? (agent_point ? 1.f : -1.f) : 0.f;
+    const bool dn = sa == kMaxScore || so == kMaxScore || e.left == 0;
+    const bool fin = ev && dn;
+    tally.episodes += fin ? 1 : 0;
+    tally.sum_return += fin ? (sa - so) : 0;
+    tally.sum_length += fin ? (kMaxFrames - e.left) : 0;
+    const int episode = e.episode + (dn ? 1 : 0);
+    sa = dn ? 0 : sa;
+    so = dn ? 0 : so;
+    uint32_t o[4];
+    philox4x32_10((uint32_t)(sa + so), (uint32_t)episode, env_id, 1u, rk, o);
+    const int nvx = (o[0] & 1u) ? kVx0 : -kVx0;
+    const int nvy = (int)__umulhi(o[1], 769u) - kVySpawn;
+    if (ev) {
+        e.sa = sa; e.so = so; e.episode = episode;
+        e.bx = kSpawnBx; e.by = kSpawnBy; e.vx = nvx; e.vy = nvy;
+        reward = r;
+        done = dn ? 1 : 0;
+        if (dn) { e.left = kMaxFrames; e.apy = kPadY0; e.opy = kPadY0; e.prev = 0; }
+    }
+}
+
+// One frame; all 32 lanes of the warp must call it together.
+__device__ __forceinline__ void fast_frame(FastEnv &e, int action, uint32_t env_id,
+                                           const RoundKeys &rk, Tally &tally, float &reward,
+                                           int &done)
+{
+    const int delta = action == 2 ? kAgentStep : (action == 1 ? -kAgentStep : 0);
+    e.apy = min(max(e.apy + delta, 0), kPadYMax);
+    const int d = e.by - e.opy - 1792;
+    e.opy = min(max(e.opy + min(max(d, -kOppStep), kOppStep), 0), kPadYMax);
+    e.bx += e.vx;
+    const int raw = e.by + e.vy;
+    const int a = abs(raw);
+    const int by = min(a, 2 * kBallYMax - a);
+    e.vy = (by != raw) ? -e.vy : e.vy;
+    e.by = by;
+    const bool right = e.vx > 0;
+    const int px = right ? kAgentXLo : kOppXLo;
+    const int py = right ? e.apy : e.opy;
+    const bool hit = (unsigned)(e.bx - px) < kHitXSpan &&
+                     (unsigned)(e.by - py + 511) < kHitYSpan;
+    if (__any_sync(0xffffffffu, hit)) {
+        const int s = min(abs(e.vx) + kVxInc, kVxCap);
+        const int nvx = right ? -s : s;
+        const int dpx = ((e.by + 256) >> 8) - ((py + 2048) >> 8);
+        const int nvy = min(max(e.vy + 16 * dpx, -kVyCap), kVyCap);
+        e.vx = hit ? nvx : e.vx;
+        e.vy = hit ? nvy : e.vy;
+    }
+    e.left -= 1;
+    const bool out = (unsigned)e.bx > (unsigned)kCourtW;
+    const bool ev = out || e.left == 0;
+    reward = 0.f;
+    done = 0;
+    if (__any_sync(0xffffffffu, ev)) fast_event(e, ev, out, env_id, rk, tally, reward, done);
+}
+
+// Philox4x32-10 advanced a few rounds at a time, so that the block for the next
+// four steps can be interleaved with the physics of the current four.
+struct PhiloxPipe {
+    uint32_t c0, c1, c2, c3;
+};
+
+__device__ __forceinline__ void philox_start(PhiloxPipe &p, unsigned long long group, uint32_t env_id)
+{
+    p.c0 = (uint32_t)group; p.c1 = env_id; p.c2 = (uint32_t)(group >> 32); p.c3 = 0u;
+}
+
+template <int R0, int R1>
+__device__ __forceinline__ void philox_rounds(PhiloxPipe &p, const RoundKeys &rk)
+{
+#pragma unroll
+    for (int r = R0; r < R1; ++r) {
+        const uint64_t p0 = (uint64_t)kPhiloxM0 * p.c0;
+        const uint64_t p1 = (uint64_t)kPhiloxM1 * p.c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ p.c1 ^ rk.k[2 * r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ p.c3 ^ rk.k[2 * r + 1];
+        p.c1 = (uint32_t)p1;
+        p.c3 = (uint32_t)p0;
+        p.c0 = n0;
+        p.c2 = n2;
+    }
+}
+
 // ---- observations -----------------------------------------------------------------
 // float32(v) is exact (|v| < 2^24); one round-to-nearest multiply by
 // float32(1/40960) = 0x37CCCCCD.  Never a division, never fused.

@@ -142,6 +142,43 @@ def test_huge_step_counter_keys_philox_with_all_64_bits(torch):
     assert_state_equal(env, ora)
 
 
+@pytest.mark.parametrize("n", [16, 48, 64, 1040, 4096])
+@pytest.mark.parametrize("mode", [0, 1])
+def test_tma_path_aligned_sizes_with_auto_resets(torch, n, mode):
+    """Sizes and step counts that take the TMA-store kernel (n % 16 == 0,
+    t % 4 == 0, T % 8 == 0), including a ragged last block, from states close
+    to the episode end so that both rare paths run often; then a mix with
+    calls that fall back to the general kernel."""
+    seed = 500 + n
+    env = pong.PongEnv(n, seed)
+    ora = oracle.OraclePong(n, seed)
+    st = random_states(n, seed=n, near_end=True)
+    env.set_state(st, 4096)
+    ora.set_state(st, 4096)
+    dones = 0
+    for T in (8, 64, 16, 128, 3, 8, 1, 24, 40):
+        g = env.rollout(T, mode)
+        o = ora.rollout(T, mode)
+        assert_outputs_equal(g, o, "n %d mode %d T %d" % (n, mode, T))
+        dones += int(o[2].sum())
+    assert dones >= n
+    assert_state_equal(env, ora)
+
+
+def test_tma_path_falls_back_on_unaligned_done_pointer(torch):
+    n, T, seed = 256, 16, 77
+    env = pong.PongEnv(n, seed)
+    ora = oracle.OraclePong(n, seed)
+    obs = torch.empty((T, n, 6), dtype=torch.float32, device="cuda")
+    reward = torch.empty((T, n), dtype=torch.float32, device="cuda")
+    raw = torch.empty((T * n + 16,), dtype=torch.uint8, device="cuda")
+    done = raw[1:1 + T * n].view(T, n)
+    assert done.data_ptr() % 16 != 0
+    env.rollout(T, 0, None, obs, reward, done)
+    assert_outputs_equal((obs, reward, done), ora.rollout(T, 0))
+    assert_state_equal(env, ora)
+
+
 # ---- single-step API -------------------------------------------------------------------------
 
 def test_step_api_against_oracle(torch):
