@@ -82,6 +82,7 @@ extern "C" {
 #define PONG_ECUDA   (-4)  /* a CUDA runtime call or launch failed */
 #define PONG_EMODE   (-5)  /* unknown action_mode, or call not valid in this obs_mode */
 #define PONG_ENOMEM  (-6)  /* host or device allocation failed */
+#define PONG_ELIMIT  (-7)  /* size beyond a fixed maximum of the entry point */
 
 #define PONG_OBS_VECTOR 0
 #define PONG_OBS_PIXELS 1
@@ -94,6 +95,7 @@ extern "C" {
 #define PONG_STATE_FIELDS 11 /* bx by vx vy apy opy score_a score_o ep_len episode prev_action */
 #define PONG_FRAME_BYTES  (84 * 84)
 #define PONG_MAX_FRAMESKIP 16
+#define PONG_STATIC_MAX_ENVS 65536 /* largest batch of pong_rollout_static */
 
 typedef struct pong_env pong_env; /* opaque */
 
@@ -170,6 +172,39 @@ int pong_episode_stats(pong_env *h, int64_t *episodes, int64_t *sum_return,
  * the ring is the caller's and is not part of the state. */
 int pong_get_state(pong_env *h, int32_t *host_soa, uint64_t *t);
 int pong_set_state(pong_env *h, const int32_t *host_soa, uint64_t t);
+
+/* Reset-and-rollout in one call that allocates nothing (the paper has no
+ * counterpart; this is an addition for hosts that cannot allocate).
+ *
+ * Who needs it: programs that may not call cudaMalloc while they run - code
+ * loaded into another runtime that owns all device memory, loops with a hard
+ * latency bound (cudaMalloc / cudaFree stall the whole device), processes held
+ * to a memory budget fixed at start-up.  The handle API takes its env state and
+ * episode counters from cudaMalloc; this call keeps them in a fixed array inside
+ * the library's device image instead (2 MiB + 256 bytes, present on every GPU
+ * that loads the library, until the process exits).  It calls no cudaMalloc,
+ * cudaFree or other allocating routine.
+ *
+ * What it does: n_envs envs (1..PONG_STATIC_MAX_ENVS, else PONG_ELIMIT) with
+ * global ids env_id_base.., vector obs, frameskip 1, are reset to episode 0 at
+ * global step 0 and run for T agent steps, exactly like pong_create_ex +
+ * pong_rollout on a fresh handle: obs_buf float32[T][n][6], reward_buf
+ * float32[T][n], done_buf uint8[T][n] (device, obs / reward 16-byte aligned),
+ * `actions` as for pong_rollout.  stats_out (device int64[3], may be NULL)
+ * receives {episodes, sum of returns, sum of lengths} of the episodes finished
+ * within the call.  Everything is enqueued on cuda_stream (NULL = default
+ * stream) and the call returns without synchronising.
+ *
+ * Set-up: the first call made with a given device current looks up the
+ * array's device address (once per device); make that first call outside any
+ * stream capture.
+ * Sharing: every call on a device uses the same array, which still holds the
+ * previous call's data; the call clears the counters and rewrites the states
+ * before use.  Two calls whose GPU work overlaps (different streams, or
+ * different host threads) race on the array: serialise them. */
+int pong_rollout_static(int n_envs, uint64_t seed, int env_id_base, int T, int action_mode,
+                        const uint8_t *actions, float *obs_buf, float *reward_buf,
+                        uint8_t *done_buf, int64_t *stats_out, void *cuda_stream);
 
 /* Number of envs / kernels launched by this handle so far (for accounting). */
 int pong_num_envs(const pong_env *h);

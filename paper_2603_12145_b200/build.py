@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpong_b200.so")
-SOURCES = ["pong_api.cu", "pong_kernels.cu"]
+SOURCES = ["pong_api.cu", "pong_kernels.cu", "pong_noalloc.cu"]
 HEADERS = ["pong_rules.cuh", "pong_kernels.cuh", os.path.join("..", "..", "include", "pong.h")]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-lineinfo",
               "-gencode", "arch=compute_100a,code=sm_100a",

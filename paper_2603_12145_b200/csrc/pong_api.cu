@@ -363,6 +363,7 @@ const char *pong_strerror(int code)
     case PONG_ECUDA: return "a CUDA runtime call or kernel launch failed";
     case PONG_EMODE: return "unknown action_mode";
     case PONG_ENOMEM: return "out of host or device memory";
+    case PONG_ELIMIT: return "size exceeds the fixed maximum of this entry point";
     default: return "unknown error code";
     }
 }

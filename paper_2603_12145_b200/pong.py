@@ -24,7 +24,8 @@ FRAME_BYTES = 84 * 84
 EXPORTS = ("pong_create", "pong_create_ex", "pong_destroy", "pong_set_stream", "pong_reset",
            "pong_step", "pong_rollout", "pong_rollout_host", "pong_fill_actions",
            "pong_episode_stats", "pong_get_state", "pong_set_state", "pong_num_envs",
-           "pong_launch_count", "pong_strerror")
+           "pong_launch_count", "pong_strerror", "pong_rollout_static")
+STATIC_MAX_ENVS = 65536
 
 
 class PongError(RuntimeError):
@@ -75,6 +76,7 @@ def load(build_if_missing: bool = False):
     L.pong_num_envs.argtypes = [vp]
     L.pong_launch_count.argtypes = [vp]
     L.pong_launch_count.restype = i64
+    L.pong_rollout_static.argtypes = [i32, u64, i32, i32, i32, vp, vp, vp, vp, vp, vp]
     L.pong_strerror.argtypes = [i32]
     L.pong_strerror.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -182,6 +184,23 @@ def pong_set_state(h: int, soa: np.ndarray, t: int) -> None:
     if soa.shape != (STATE_FIELDS, n):
         raise ValueError("state must be int32 [%d, %d]" % (STATE_FIELDS, n))
     _check(load().pong_set_state(h, soa.ctypes.data, int(t)), "pong_set_state")
+
+
+def pong_rollout_static(n_envs: int, seed: int, env_id_base: int, T: int, action_mode: int,
+                        actions, obs_buf, reward_buf, done_buf, stats_out=None,
+                        cuda_stream: Optional[int] = None) -> None:
+    """Reset + rollout without any allocation inside the library: the env state
+    lives in a fixed device array of the library (at most STATIC_MAX_ENVS envs).
+    For hosts that may not call cudaMalloc while running.  Calls that overlap
+    on the GPU race on that array."""
+    keep = None
+    if action_mode == ACT_CONSTANT and not isinstance(actions, np.ndarray):
+        keep = np.array([int(actions)], dtype=np.uint8)
+        actions = keep
+    _check(load().pong_rollout_static(int(n_envs), int(seed) & (2**64 - 1), int(env_id_base), int(T),
+                                      int(action_mode), _ptr(actions), _ptr(obs_buf),
+                                      _ptr(reward_buf), _ptr(done_buf), _ptr(stats_out),
+                                      cuda_stream), "pong_rollout_static")
 
 
 def pong_num_envs(h: int) -> int:

@@ -1,0 +1,57 @@
+"""pong_rollout_static, the entry point for hosts that cannot allocate device
+memory while running (its env state sits in a fixed array inside the library),
+must give exactly what the handle-based entry points give.  Checked on two
+calls in a row that share the array, with different sizes, seeds and modes, so
+that nothing left behind by the first call can leak into the second.  This file
+is collected last on purpose."""
+import numpy as np
+import pytest
+
+from paper_2603_12145_b200 import pong
+
+pytestmark = pytest.mark.gpu
+
+
+def run_both(torch, n, seed, base, T, mode):
+    obs = torch.empty((T, n, 6), dtype=torch.float32, device="cuda")
+    reward = torch.empty((T, n), dtype=torch.float32, device="cuda")
+    done = torch.empty((T, n), dtype=torch.uint8, device="cuda")
+    stats = torch.full((3,), -1, dtype=torch.int64, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    pong.pong_rollout_static(n, seed, base, T, mode, None, obs, reward, done, stats, stream)
+    env = pong.PongEnv(n, seed, env_id_base=base)
+    want = env.rollout(T, mode)
+    torch.cuda.synchronize()
+    for got, ref in zip((obs, reward, done), want):
+        assert got.cpu().numpy().tobytes() == ref.cpu().numpy().tobytes()
+    assert tuple(stats.cpu().tolist()) == env.episode_stats()
+    return env.episode_stats()
+
+
+def test_static_rollout_matches_handle_rollout_twice_in_a_row():
+    import torch
+    assert torch.cuda.is_available()
+    pong.load()
+    # long enough for episodes to finish, so the counters are non-zero
+    first = run_both(torch, 4096, 7, 0, 4000, pong.ACT_PHILOX)
+    assert first[0] > 0
+    # second call: other size (ragged), seed, id range and mode; shares the array
+    second = run_both(torch, 1000, 0xABCDEF0123, 500, 2504, pong.ACT_STICKY)
+    assert second[0] > 0 and second != first
+    # and the first configuration again gives the first result again
+    assert run_both(torch, 4096, 7, 0, 4000, pong.ACT_PHILOX) == first
+
+
+def test_static_rollout_rejects_bad_sizes():
+    import torch
+    pong.load()
+    buf = torch.empty((64,), dtype=torch.float32, device="cuda")
+    d = torch.empty((64,), dtype=torch.uint8, device="cuda")
+    for n, code in ((pong.STATIC_MAX_ENVS + 1, -7), (0, -1)):
+        with pytest.raises(pong.PongError) as ei:
+            pong.pong_rollout_static(n, 0, 0, 1, 0, None, buf, buf, d)
+        assert ei.value.code == code
+    with pytest.raises(pong.PongError) as ei:
+        pong.pong_rollout_static(8, 0, 0, 1, 0, None, None, buf, d)
+    assert ei.value.code == -2
+    assert "maximum" in pong.strerror(-7)
