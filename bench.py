@@ -3,11 +3,13 @@
 fraction of the HBM roofline.
 
 One "step" of this benchmark is one fused rollout launch over the whole batch:
-N = 65,536 envs x T = 128 agent steps with in-kernel Philox actions, vector
-observations float32[T,N,6] plus reward and done buffers, and the episode
+by default N = 65,536 envs x T = 128 agent steps with in-kernel Philox actions,
+vector observations float32[T,N,6] plus reward and done buffers, and the episode
 statistics reduction, i.e. 8,388,608 env-steps and 243 MB written per step.
+--workload selects one of the other configurations instead.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+                    [--workload rollout65k|rollout1m|pixels16k|step4096|small64]
 
 Prints one JSON line (rank 0).  With --gpus N > 1 it must be launched with
 torchrun, one rank per GPU; each rank simulates its own 65,536 envs (global env
@@ -27,21 +29,41 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-N_ENVS = 65536
-T_STEPS = 128
 SEED = 0
 METRIC = "env-steps/sec on 1 B200 and achieved HBM GB/s fraction of roofline"
 UNIT = "env-steps/s"
-WORKLOAD = "fused vector-obs rollout, N=65536 envs, T=128 steps per launch, in-kernel Philox actions"
-# Algorithmic bytes per env-step: obs 24 + reward 4 + done 1 written, plus the
-# 32-byte state read and written once per launch (64 / T).
-BYTES_PER_ENV_STEP = 29.0 + 64.0 / T_STEPS
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the rollout
-# kernel from an ncu capture of this workload (see profiles/); None when the
-# kernel has changed since the counters were taken.
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+# The default workload ("rollout65k") is the one the headline metric is quoted
+# on; the others are the remaining configurations, selectable with --workload.
+# bytes: algorithmic bytes per env-step = outputs written per agent step plus the
+# 32-byte state read and written once per launch (64 / T); the single-step API
+# also reads one action byte.
+# traffic: dram__bytes_read.sum + dram__bytes_write.sum of one launch from an ncu
+# capture of that workload (profiles/), None if not captured for the current kernel.
+WORKLOADS = {
+    "rollout65k": dict(
+        name="fused vector-obs rollout, N=65536 envs, T=128 steps per launch, in-kernel Philox actions",
+        n=65536, T=128, mode=0, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 128,
+        kernel="k_rollout_vector_tma", traffic=None),
+    "rollout1m": dict(
+        name="fused vector-obs rollout, N=1048576 envs, T=32 steps per launch, in-kernel Philox sticky actions",
+        n=1048576, T=32, mode=1, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 32,
+        kernel="k_rollout_vector_tma", traffic=None),
+    "pixels16k": dict(
+        name="pixel-obs rollout, N=16384 envs, T=64 agent steps per launch, frameskip 4, 4-frame ring uint8[N,4,84,84]",
+        n=16384, T=64, mode=0, obs_mode=1, frameskip=4, bytes=7056.0 + 5.0 + 64.0 / 64,
+        kernel="k_rollout_pixels_x4", traffic=None),
+    "step4096": dict(
+        name="single-step API pong_step, N=4096 envs, one agent step per launch, actions from a device buffer",
+        n=4096, T=1, mode=2, obs_mode=0, frameskip=1, bytes=94.0,
+        kernel="k_rollout_vector", traffic=None),
+    "small64": dict(
+        name="fused vector-obs rollout, N=64 envs, T=2000 steps per launch, in-kernel Philox actions",
+        n=64, T=2000, mode=0, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 2000,
+        kernel="k_rollout_vector_tma", traffic=None),
+}
 
 
 def measured_peak():
@@ -124,46 +146,58 @@ def physical_gpu_index(local):
     return local
 
 
-def cpu_oracle_rate(budget_s, n_sample=8192, min_reps=1):
-    """Env-steps/s of the CPU oracle, as it stands, on one host thread: envs
-    0..n_sample-1 of the same workload, T=128 steps per call, repeated until the
-    time budget is used."""
+def oracle_sample(w):
+    """The oracle on a bounded sample of a workload: its first envs, same T,
+    action mode, obs mode and frameskip.  Returns (oracle, n_sample, call)."""
+    import numpy as np
     import oracle
-    o = oracle.OraclePong(n_sample, SEED)
-    o.rollout(T_STEPS, 0)                       # warm-up (page-in, first touch)
+    from paper_2603_12145_b200.inputs import explicit_actions
+    n_sample = min(w["n"], 256 if w["obs_mode"] == 1 else 8192)
+    o = oracle.OraclePong(n_sample, SEED, obs_mode=w["obs_mode"], frameskip=w["frameskip"])
+    if w["mode"] == 2:
+        acts = explicit_actions(w["T"], n_sample, seed=SEED)
+        return o, n_sample, (lambda: o.rollout(w["T"], 2, acts))
+    return o, n_sample, (lambda: o.rollout(w["T"], w["mode"]))
+
+
+def cpu_oracle_rate(w, budget_s):
+    """Env-steps/s of the CPU oracle, as it stands, on one host thread, repeated
+    until the time budget is used."""
+    o, n_sample, call = oracle_sample(w)
+    call()                                      # warm-up (page-in, first touch)
     steps, reps, t0 = 0, 0, time.perf_counter()
     while True:
-        o.rollout(T_STEPS, 0)
-        steps += n_sample * T_STEPS
+        call()
+        steps += n_sample * w["T"]
         reps += 1
         dt = time.perf_counter() - t0
-        if reps >= min_reps and dt >= budget_s:
+        if dt >= budget_s:
             break
-    return steps / dt, reps, dt
+    return steps / dt, reps, dt, n_sample
 
 
 def run_reference(args, rank):
     if rank != 0:
         return
-    n_sample = 8192
-    import oracle
-    o = oracle.OraclePong(n_sample, SEED)
-    for _ in range(max(args.warmup, 1)):
-        o.rollout(T_STEPS, 0)
-    # each step: T=128 oracle steps of the first 8192 envs of the workload;
-    # cap the run at about two minutes whatever --steps says
-    k = max(1, min(args.steps, 200))
+    w = WORKLOADS[args.workload]
+    WORKLOAD = w["name"]
+    o, n_sample, call = oracle_sample(w)
+    for _ in range(max(min(args.warmup, 5), 1)):
+        call()
+    # each step: one oracle call (T agent steps) on the first n_sample envs of the
+    # workload; the run is capped at about two minutes whatever --steps says
+    k = args.steps if args.steps > 0 else 50
     t0 = time.perf_counter()
     done_steps = 0
     for i in range(k):
-        o.rollout(T_STEPS, 0)
+        call()
         done_steps += 1
         if time.perf_counter() - t0 > 120.0:
             break
     dt = time.perf_counter() - t0
-    value = done_steps * n_sample * T_STEPS / dt
+    value = done_steps * n_sample * w["T"] / dt
     sample = "envs 0..%d of the workload, T=%d per step, %d steps, single thread" % (
-        n_sample - 1, T_STEPS, done_steps)
+        n_sample - 1, w["T"], done_steps)
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": done_steps, "warmup": max(args.warmup, 1), "ms_per_step": dt / done_steps * 1e3,
@@ -177,9 +211,10 @@ def run_reference(args, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5000)
+    ap.add_argument("--steps", type=int, default=0, help="timed launches (default: per workload)")
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--workload", default="rollout65k", choices=sorted(WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     args = ap.parse_args()
@@ -194,7 +229,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2603_12145_b200 import pong
+    from paper_2603_12145_b200 import pong, sharding
     from paper_2603_12145_b200.inputs import explicit_actions
 
     if not torch.cuda.is_available():
@@ -206,13 +241,38 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     pong.load()
-    warmup = max(args.warmup, 3)
-    steps = max(args.steps, 1)
 
-    env = pong.PongEnv(N_ENVS, SEED, env_id_base=rank * N_ENVS)
-    obs = torch.empty((T_STEPS, N_ENVS, 6), dtype=torch.float32, device="cuda")
-    reward = torch.empty((T_STEPS, N_ENVS), dtype=torch.float32, device="cuda")
-    done = torch.empty((T_STEPS, N_ENVS), dtype=torch.uint8, device="cuda")
+    w = WORKLOADS[args.workload]
+    N, T, mode = w["n"], w["T"], w["mode"]
+    pixels = w["obs_mode"] == 1
+    env_steps_per_launch = N * T
+    warmup = max(args.warmup, 3)
+    # default launch count: about 0.3 s of timed work
+    default_steps = {"rollout65k": 5000, "rollout1m": 1500, "pixels16k": 200, "step4096": 20000,
+                     "small64": 300}[args.workload]
+    steps = args.steps if args.steps > 0 else default_steps
+
+    env_id_base, _ = sharding.shard(rank, world, N)
+    env = pong.PongEnv(N, SEED, obs_mode=w["obs_mode"], frameskip=w["frameskip"],
+                       env_id_base=env_id_base)
+    obs = env.ring if pixels else torch.empty((T, N, 6), dtype=torch.float32, device="cuda")
+    reward = torch.empty((T, N), dtype=torch.float32, device="cuda")
+    done = torch.empty((T, N), dtype=torch.uint8, device="cuda")
+    acts_np = explicit_actions(T, N, seed=SEED)
+    acts_d = torch.from_numpy(acts_np).cuda() if mode == 2 else None
+    l2_note = ("each step writes %.0f MB of outputs, larger than the 126 MB L2; no flush"
+               % (env_steps_per_launch * w["bytes"] / 1e6))
+    flush = None
+    if env_steps_per_launch * w["bytes"] < 200e6:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        l2_note = "outputs smaller than L2: a 256 MB buffer is rewritten before the timed region only " \
+                  "(launch-latency-bound workload; flushing between launches would time the flush)"
+
+    def launch():
+        if args.workload == "step4096":
+            env.step(acts_d[0], obs[0], reward[0], done[0])
+        else:
+            env.rollout(T, mode, acts_d, obs, reward, done)
 
     def barrier():
         if world > 1:
@@ -222,7 +282,9 @@ def main():
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
     for _ in range(warmup):
-        env.rollout(T_STEPS, pong.ACT_PHILOX, None, obs, reward, done)
+        launch()
+    if flush is not None:
+        flush.fill_(1)
     barrier()
 
     # ---- device-resident timing: K launches, CUDA events on the launching stream
@@ -234,7 +296,7 @@ def main():
     for s in range(n_seg):
         lo, hi = steps * s // n_seg, steps * (s + 1) // n_seg
         for _ in range(hi - lo):
-            env.rollout(T_STEPS, pong.ACT_PHILOX, None, obs, reward, done)
+            launch()
         marks[s + 1].record()
     torch.cuda.synchronize()
     w1 = time.perf_counter()
@@ -244,42 +306,36 @@ def main():
     seg_rates = []
     for s in range(n_seg):
         k = steps * (s + 1) // n_seg - steps * s // n_seg
-        seg_rates.append(k * N_ENVS * T_STEPS / (marks[s].elapsed_time(marks[s + 1]) * 1e-3))
-    if world > 1:
-        tmax = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms_total = float(tmax.item())
-    stats = env.episode_stats()
+        seg_rates.append(k * env_steps_per_launch / (marks[s].elapsed_time(marks[s + 1]) * 1e-3))
+    ms_total = sharding.max_over_ranks(ms_total, device="cuda")
+    stats = sharding.sum_stats(env.episode_stats(), device="cuda")
 
     # ---- end to end: host buffers in, host buffers out, through pong_rollout_host
     e2e_steps = max(args.e2e_steps, 1)
-    acts_h = torch.from_numpy(explicit_actions(T_STEPS, N_ENVS, seed=SEED)).pin_memory()
-    obs_h = torch.empty((T_STEPS, N_ENVS, 6), dtype=torch.float32).pin_memory()
-    rew_h = torch.empty((T_STEPS, N_ENVS), dtype=torch.float32).pin_memory()
-    done_h = torch.empty((T_STEPS, N_ENVS), dtype=torch.uint8).pin_memory()
+    acts_h = torch.from_numpy(acts_np).pin_memory()
+    obs_h = (torch.zeros((N, 4, 84, 84), dtype=torch.uint8) if pixels
+             else torch.empty((T, N, 6), dtype=torch.float32)).pin_memory()
+    rew_h = torch.empty((T, N), dtype=torch.float32).pin_memory()
+    done_h = torch.empty((T, N), dtype=torch.uint8).pin_memory()
     env._stream()
     for _ in range(2):
-        pong.pong_rollout_host(env.h, T_STEPS, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
+        pong.pong_rollout_host(env.h, T, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
     barrier()
     e0 = time.perf_counter()
     for _ in range(e2e_steps):
-        pong.pong_rollout_host(env.h, T_STEPS, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
+        pong.pong_rollout_host(env.h, T, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - e0
-    if world > 1:
-        tmax = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_s = float(tmax.item())
+    e2e_s = sharding.max_over_ranks(e2e_s, device="cuda")
     sampler.stop()
     barrier()
 
-    env_steps_per_launch = N_ENVS * T_STEPS
     value = world * steps * env_steps_per_launch / (ms_total * 1e-3)
     peak, peak_kind = measured_peak()
     kernel_ms = ms_total / steps
-    achieved = env_steps_per_launch * BYTES_PER_ENV_STEP / (kernel_ms * 1e-3) / 1e9
-    h2d = acts_h.numel()
-    d2h = obs_h.numel() * 4 + rew_h.numel() * 4 + done_h.numel()
+    achieved = env_steps_per_launch * w["bytes"] / (kernel_ms * 1e-3) / 1e9
+    h2d = acts_h.numel() + (obs_h.numel() if pixels else 0)
+    d2h = obs_h.numel() * obs_h.element_size() + rew_h.numel() * 4 + done_h.numel()
 
     if rank == 0:
         mean = sum(seg_rates) / len(seg_rates)
@@ -289,19 +345,19 @@ def main():
             "warmup": warmup, "ms_per_step": kernel_ms, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
             "config": {
-                "workload": WORKLOAD, "n_envs_per_gpu": N_ENVS, "T": T_STEPS, "seed": SEED,
-                "env_steps_per_step": env_steps_per_launch,
-                "l2": "each step writes 243 MB of outputs, larger than the 126 MB L2; no flush",
+                "workload": w["name"], "workload_key": args.workload, "n_envs_per_gpu": N, "T": T,
+                "frameskip": w["frameskip"], "seed": SEED, "env_steps_per_step": env_steps_per_launch,
+                "l2": l2_note,
                 "parallelism": "env shards per GPU, no collective" if world > 1 else "single GPU",
             },
             "roofline": {
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
-                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
-                "algorithmic_bytes_per_launch": env_steps_per_launch * BYTES_PER_ENV_STEP,
-                "bytes_per_env_step": BYTES_PER_ENV_STEP,
+                "traffic": w["traffic"],
+                "algorithmic_bytes_per_launch": env_steps_per_launch * w["bytes"],
+                "bytes_per_env_step": w["bytes"],
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "kernel": "k_rollout_vector_tma", "kernel_ms": kernel_ms,
+                "kernel": w["kernel"], "kernel_ms": kernel_ms,
             },
             "e2e": {"value": world * e2e_steps * env_steps_per_launch / e2e_s, "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
@@ -312,12 +368,12 @@ def main():
             "episode_stats": {"episodes": stats[0], "sum_return": stats[1], "sum_length": stats[2]},
         }
         if world == 1:
-            rate, reps, dt = cpu_oracle_rate(args.cpu_seconds)
+            rate, reps, dt, n_sample = cpu_oracle_rate(w, args.cpu_seconds)
             line["cpu_baseline"] = {
                 "value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
                 "host_cores": os.cpu_count(),
-                "sample": "envs 0..8191 of the workload, T=128 per call, %d calls, %.1f s, "
-                          "single thread" % (reps, dt)}
+                "sample": "envs 0..%d of the workload, T=%d per call, %d calls, %.1f s, "
+                          "single thread" % (n_sample - 1, T, reps, dt)}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -13,6 +13,10 @@
 //   k_rollout_pixels   one thread per env for the physics, one warp per frame
 //                      for the rasteriser; frames are staged in shared memory
 //                      and leave through bulk async copies (16-byte granules)
+//   k_rollout_pixels_x4  the same for aligned calls (t % 4 == 0, T % 4 == 0): four
+//                      agent steps at a time, so that an env's whole 4-slot ring
+//                      (28,224 contiguous bytes) is painted in shared memory and
+//                      leaves as one bulk copy
 //   k_fill_actions     action bytes that reproduce the Philox modes
 //
 // No kernel waits on another block, on a flag or on an mbarrier; the only
@@ -470,22 +474,121 @@ __global__ void __launch_bounds__(kPixThreads) k_rollout_pixels(const __grid_con
     flush_tally(tally, a.stats);
 }
 
+// Four agent steps per pass.  Steps 4k .. 4k+3 write ring slots 0 .. 3, and a step
+// that ends an episode writes its reset frame to all four slots, so after the four
+// steps slot s holds the frame of the last step j >= s with j == s or done(j).
+// That is worked out per env on the geometry words; then each env's ring is painted
+// once and stored as one contiguous 28,224-byte bulk copy: the same bytes per agent
+// step as the frame-at-a-time kernel, but every DRAM page is written in one go.
+constexpr int kPix4Warps = 3;
+constexpr int kPix4Threads = kPix4Warps * 32;
+constexpr int kPix4Bufs = 2;  // staged rings per warp
+constexpr int kRingBytes = kStack * kFrameBytes;
+constexpr int kPix4SmemBytes = kPix4Warps * kPix4Bufs * kRingBytes + kPix4Threads * 16;
+
+template <int MODE>
+__global__ void __launch_bounds__(kPix4Threads) k_rollout_pixels_x4(const __grid_constant__ LaunchArgs a,
+                                                                   const int envs_per_block)
+{
+    extern __shared__ __align__(128) uint8_t smem[];
+    uint8_t *rings = smem;
+    uint4 *geom = reinterpret_cast<uint4 *>(smem + kPix4Warps * kPix4Bufs * kRingBytes);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int first = blockIdx.x * envs_per_block;
+    const int count = min(envs_per_block, a.n - first);
+    const bool has_env = tid < count;
+    const int n = first + tid;
+    const uint32_t env_id = a.env_id_base + (uint32_t)n;
+
+    Env e = {};
+    Tally tally = {0, 0, 0};
+    if (has_env) load_env(e, a.plane0, a.plane1, n);
+    unsigned round = 0;
+
+    for (int t = 0; t < a.T; t += 4) {
+        if (has_env) {
+            uint32_t w[4] = {0u, 0u, 0u, 0u};
+            if (MODE <= 1) action_words((a.t0 + (unsigned long long)t) >> 2, env_id, a.rk, w);
+            uint32_t g[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const size_t o = (size_t)(t + j) * (size_t)a.n + (size_t)n;
+                const int action = pick_action<MODE>(w[j], e, MODE == 2 ? a.actions + o : nullptr,
+                                                     a.const_action);
+                bool done;
+                const int r = agent_step<0>(e, action, a.frameskip, env_id, a.rk, tally, done);
+                a.reward[o] = (float)r;
+                a.done[o] = done ? 1 : 0;
+                const uint32_t gj = pack_geometry(e);
+                g[j] = gj;
+                if (done) {
+#pragma unroll
+                    for (int s = 0; s < 4; ++s) g[s] = gj;
+                }
+            }
+            geom[tid] = make_uint4(g[0], g[1], g[2], g[3]);
+        }
+        __syncthreads();
+        for (int le = warp; le < count; le += kPix4Warps) {
+            uint8_t *buf = rings + (warp * kPix4Bufs + (round % kPix4Bufs)) * kRingBytes;
+            ++round;
+            if (lane == 0) bulk_wait_read<kPix4Bufs - 1>();
+            __syncwarp();
+            const uint4 gq = geom[le];
+            render_frame(buf, gq.x, lane);
+            render_frame(buf + kFrameBytes, gq.y, lane);
+            render_frame(buf + 2 * kFrameBytes, gq.z, lane);
+            render_frame(buf + 3 * kFrameBytes, gq.w, lane);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                bulk_store(a.ring + (size_t)(first + le) * kRingBytes, buf, kRingBytes);
+                bulk_commit();
+            }
+        }
+        __syncthreads();
+    }
+    if (lane == 0) bulk_wait_read<0>();
+    if (has_env) store_env(e, a.plane0, a.plane1, n);
+    flush_tally(tally, a.stats);
+}
+
 // Envs per block so that the grid is a whole number of waves over the SMs
 // (two resident blocks per SM) while no block gets more envs than threads.
-static int pixel_envs_per_block(int n, int sm_count)
+static int pixel_envs_per_block(int n, int sm_count, int max_per_block)
 {
     for (int k = 2;; k += 2) {
         const int slots = sm_count * k;
         const int per = (n + slots - 1) / slots;
-        if (per <= kPixThreads) return per;
+        if (per <= max_per_block) return per;
     }
 }
 
 cudaError_t launch_rollout_pixels(const LaunchArgs &a, int sm_count, cudaStream_t s)
 {
-    const int per = pixel_envs_per_block(a.n, sm_count);
-    const int grid = (a.n + per - 1) / per;
     cudaError_t err = cudaSuccess;
+    if (a.t0 % 4 == 0 && a.T % 4 == 0) {
+        const int per = pixel_envs_per_block(a.n, sm_count, kPix4Threads);
+        const int grid = (a.n + per - 1) / per;
+#define PONG_PIX4(M)                                                                                \
+    do {                                                                                            \
+        err = cudaFuncSetAttribute(k_rollout_pixels_x4<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                   kPix4SmemBytes);                                                 \
+        if (err != cudaSuccess) return err;                                                         \
+        k_rollout_pixels_x4<M><<<grid, kPix4Threads, kPix4SmemBytes, s>>>(a, per);                  \
+    } while (0)
+        switch (a.action_mode) {
+        case 0: PONG_PIX4(0); break;
+        case 1: PONG_PIX4(1); break;
+        case 2: PONG_PIX4(2); break;
+        default: PONG_PIX4(3); break;
+        }
+#undef PONG_PIX4
+        return cudaGetLastError();
+    }
+    const int per = pixel_envs_per_block(a.n, sm_count, kPixThreads);
+    const int grid = (a.n + per - 1) / per;
 #define PONG_PIX(M)                                                                              \
     do {                                                                                         \
         err = cudaFuncSetAttribute(k_rollout_pixels<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, \

@@ -311,6 +311,40 @@ def test_pixel_rollout_and_step_against_oracle(torch, n):
     assert same(cpu(env.reset()), ora.reset())
 
 
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
+def test_pixel_four_step_path_with_resets_inside_a_pass(torch, mode):
+    """Aligned calls (t % 4 == 0, T % 4 == 0) take the kernel that paints a whole
+    4-slot ring per pass; episode ends in the middle of a pass must leave every
+    slot as the frame-at-a-time definition does."""
+    n, seed = 203, 77
+    env = pong.PongEnv(n, seed, obs_mode=1, frameskip=4)
+    ora = oracle.OraclePong(n, seed, obs_mode=1, frameskip=4)
+    st = random_states(n, seed=9, near_end=True)
+    st[8] = 9999 - (np.arange(n) % 40)          # episodes end at every phase of a pass
+    env.set_state(st, 64)
+    ora.set_state(st, 64)
+    dones = 0
+    for k, T in enumerate((4, 8, 4, 12, 4, 4, 64)):
+        if mode == 2:
+            acts = explicit_actions(T, n, seed=k, repeat_fraction=0.2)
+            g = env.rollout(T, 2, torch.from_numpy(acts).cuda())
+            o = ora.rollout(T, 2, acts)
+        elif mode == 3:
+            g = env.rollout(T, 3, k % 3)
+            o = ora.rollout(T, 3, k % 3)
+        else:
+            g = env.rollout(T, mode)
+            o = ora.rollout(T, mode)
+        assert_outputs_equal(g, o, "x4 mode %d T %d" % (mode, T))
+        dones += int(o[2].sum())
+    assert dones >= n
+    assert_state_equal(env, ora)
+    # then unaligned calls (frame-at-a-time kernel) and back
+    for T in (3, 1, 4, 8):
+        assert_outputs_equal(env.rollout(T, 0), ora.rollout(T, 0), "mixed T %d" % T)
+    assert_state_equal(env, ora)
+
+
 def test_pixel_frameskip_one_and_constant_action(torch):
     n, seed = 50, 8
     env = pong.PongEnv(n, seed, obs_mode=1, frameskip=1)
