@@ -5,8 +5,8 @@
 //   k_rollout_vector   one thread per env, state in registers across T steps,
 //                      streams obs / reward / done to HBM with per-thread stores
 //                      (any n, T, frameskip and action mode)
-//   k_rollout_vector_tma  the same rollout for the common case (Philox actions,
-//                      frameskip 1, aligned n / t / T): outputs are staged in shared
+//   k_rollout_vector_tma  the same rollout for the common case (frameskip 1,
+//                      aligned n / t / T, any action mode): outputs are staged in shared
 //                      memory 8 steps at a time and leave through TMA tensor stores,
 //                      the Philox block of the next four steps is interleaved with
 //                      the physics of the current four, rare paths are warp-uniform
@@ -220,9 +220,11 @@ __global__ void __launch_bounds__(kTmaBlock) k_rollout_vector_tma(const __grid_c
     // Philox block of the first four steps: independent of the state, so it runs
     // before the wait on the previous kernel.
     unsigned long long g = a.t0 >> 2;
-    PhiloxPipe pipe;
-    philox_start(pipe, g, env_id);
-    philox_rounds<0, 10>(pipe, a.rk);
+    PhiloxPipe pipe = {0u, 0u, 0u, 0u};
+    if (MODE <= 1) {
+        philox_start(pipe, g, env_id);
+        philox_rounds<0, 10>(pipe, a.rk);
+    }
 
     grid_dependency_wait();
     FastEnv e;
@@ -233,25 +235,42 @@ __global__ void __launch_bounds__(kTmaBlock) k_rollout_vector_tma(const __grid_c
     }
     grid_dependency_launch();
 
+    const uint8_t *act = MODE == 2 ? a.actions + n : nullptr;
+    const size_t act_stride = (size_t)a.n;
     int buf = 0;
     for (int t = 0; t < a.T; t += kTmaStage) {
+        // explicit actions of this stage: eight coalesced byte loads issued together,
+        // their latency hidden behind the wait below
+        uint32_t abyte[kTmaStage];
+        if (MODE == 2) {
+#pragma unroll
+            for (int s = 0; s < kTmaStage; ++s) abyte[s] = act[(size_t)s * act_stride];
+            act += (size_t)kTmaStage * act_stride;
+        }
         // the store that last read this buffer is the older of the two in flight
         if (tid == 0) bulk_wait_read<1>();
         __syncthreads();
 #pragma unroll
         for (int q = 0; q < kTmaStage / 4; ++q) {
             const uint32_t w[4] = {pipe.c0, pipe.c1, pipe.c2, pipe.c3};
-            ++g;
-            philox_start(pipe, g, env_id);
+            if (MODE <= 1) {
+                ++g;
+                philox_start(pipe, g, env_id);
+            }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                if (j == 0) philox_rounds<0, 3>(pipe, a.rk);
-                if (j == 1) philox_rounds<3, 6>(pipe, a.rk);
-                if (j == 2) philox_rounds<6, 8>(pipe, a.rk);
-                if (j == 3) philox_rounds<8, 10>(pipe, a.rk);
+                if (MODE <= 1) {
+                    if (j == 0) philox_rounds<0, 3>(pipe, a.rk);
+                    if (j == 1) philox_rounds<3, 6>(pipe, a.rk);
+                    if (j == 2) philox_rounds<6, 8>(pipe, a.rk);
+                    if (j == 3) philox_rounds<8, 10>(pipe, a.rk);
+                }
                 const int s = q * 4 + j;
-                int action = uniform_action(w[j]);
-                if (MODE == 1) action = sticky_repeat(w[j]) ? e.prev : action;
+                int action;
+                if (MODE == 0) action = uniform_action(w[j]);
+                else if (MODE == 1) action = sticky_repeat(w[j]) ? e.prev : uniform_action(w[j]);
+                else if (MODE == 2) action = decode_action_byte(abyte[s], e.prev);
+                else action = a.const_action;
                 e.prev = action;
                 float r;
                 int dn;
@@ -326,7 +345,7 @@ static bool encode_rows(TensorMapEncodeFn enc, CUtensorMap *m, CUtensorMapDataTy
 // if it does not, so that the caller uses the general kernel.
 static bool try_launch_vector_tma(const LaunchArgs &a, cudaStream_t s, cudaError_t *err)
 {
-    if (a.action_mode > 1 || a.frameskip != 1) return false;
+    if (a.frameskip != 1) return false;
     if (a.n % 16 != 0 || a.t0 % 4 != 0 || a.T % kTmaStage != 0) return false;
     const uintptr_t bases = reinterpret_cast<uintptr_t>(a.obs) | reinterpret_cast<uintptr_t>(a.reward) |
                             reinterpret_cast<uintptr_t>(a.done);
@@ -351,10 +370,12 @@ static bool try_launch_vector_tma(const LaunchArgs &a, cudaStream_t s, cudaError
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (a.action_mode == 0)
-        *err = cudaLaunchKernelEx(&cfg, k_rollout_vector_tma<0>, a, maps);
-    else
-        *err = cudaLaunchKernelEx(&cfg, k_rollout_vector_tma<1>, a, maps);
+    switch (a.action_mode) {
+    case 0: *err = cudaLaunchKernelEx(&cfg, k_rollout_vector_tma<0>, a, maps); break;
+    case 1: *err = cudaLaunchKernelEx(&cfg, k_rollout_vector_tma<1>, a, maps); break;
+    case 2: *err = cudaLaunchKernelEx(&cfg, k_rollout_vector_tma<2>, a, maps); break;
+    default: *err = cudaLaunchKernelEx(&cfg, k_rollout_vector_tma<3>, a, maps); break;
+    }
     return true;
 }
 

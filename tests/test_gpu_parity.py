@@ -143,7 +143,7 @@ def test_huge_step_counter_keys_philox_with_all_64_bits(torch):
 
 
 @pytest.mark.parametrize("n", [16, 48, 64, 1040, 4096])
-@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("mode", [0, 1, 2, 3])
 def test_tma_path_aligned_sizes_with_auto_resets(torch, n, mode):
     """Sizes and step counts that take the TMA-store kernel (n % 16 == 0,
     t % 4 == 0, T % 8 == 0), including a ragged last block, from states close
@@ -156,9 +156,17 @@ def test_tma_path_aligned_sizes_with_auto_resets(torch, n, mode):
     env.set_state(st, 4096)
     ora.set_state(st, 4096)
     dones = 0
-    for T in (8, 64, 16, 128, 3, 8, 1, 24, 40):
-        g = env.rollout(T, mode)
-        o = ora.rollout(T, mode)
+    for k, T in enumerate((8, 64, 16, 128, 3, 8, 1, 24, 40)):
+        if mode == 2:
+            acts = explicit_actions(T, n, seed=k, repeat_fraction=0.25, odd_codes=True)
+            g = env.rollout(T, 2, torch.from_numpy(acts).cuda())
+            o = ora.rollout(T, 2, acts)
+        elif mode == 3:
+            g = env.rollout(T, 3, (k + 1) % 3)
+            o = ora.rollout(T, 3, (k + 1) % 3)
+        else:
+            g = env.rollout(T, mode)
+            o = ora.rollout(T, mode)
         assert_outputs_equal(g, o, "n %d mode %d T %d" % (n, mode, T))
         dones += int(o[2].sum())
     assert dones >= n
