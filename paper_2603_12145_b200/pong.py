@@ -217,6 +217,8 @@ class PongEnv:
     """Owns a handle plus (optionally) torch output tensors.  Every call runs
     on torch's current CUDA stream."""
 
+    device_actions = True  # explicit action buffers must be device tensors
+
     def __init__(self, n_envs: int, seed: int, obs_mode: int = OBS_VECTOR, frameskip: int = 1,
                  env_id_base: int = 0, device: Optional[str] = None):
         import torch
