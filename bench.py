@@ -9,7 +9,8 @@ statistics reduction, i.e. 8,388,608 env-steps and 243 MB written per step.
 --workload selects one of the other configurations instead.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
-                    [--workload rollout65k|rollout1m|pixels16k|step4096|small64]
+                    [--workload rollout65k|rollout1m|pixels16k|step4096|small64|
+                                cartpole65k|cartpole1m]
 
 Prints one JSON line (rank 0).  With --gpus N > 1 it must be launched with
 torchrun, one rank per GPU; each rank simulates its own 65,536 envs (global env
@@ -39,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # on; the others are the remaining configurations, selectable with --workload.
 # bytes: algorithmic bytes per env-step = outputs written per agent step plus the
 # 32-byte state read and written once per launch (64 / T); the single-step API
-# also reads one action byte.
+# also reads one action byte.  CartPole: obs 16 + reward 4 + done 1, state 24 bytes.
 # traffic: dram__bytes_read.sum + dram__bytes_write.sum of one launch from an ncu
 # capture of that workload (profiles/), None if not captured for the current kernel.
 WORKLOADS = {
@@ -59,6 +60,14 @@ WORKLOADS = {
         name="single-step API pong_step, N=4096 envs, one agent step per launch, actions from a device buffer",
         n=4096, T=1, mode=2, obs_mode=0, frameskip=1, bytes=94.0,
         kernel="k_rollout_vector", traffic=None),
+    "cartpole65k": dict(
+        name="CartPole fused rollout, N=65536 envs, T=128 steps per launch, in-kernel Philox actions",
+        env="cartpole", n=65536, T=128, mode=0, obs_mode=0, frameskip=1, bytes=21.0 + 48.0 / 128,
+        kernel="k_cartpole_rollout", traffic=None),
+    "cartpole1m": dict(
+        name="CartPole fused rollout, N=1048576 envs, T=32 steps per launch, in-kernel Philox actions",
+        env="cartpole", n=1048576, T=32, mode=0, obs_mode=0, frameskip=1, bytes=21.0 + 48.0 / 32,
+        kernel="k_cartpole_rollout", traffic=None),
     "small64": dict(
         name="fused vector-obs rollout, N=64 envs, T=2000 steps per launch, in-kernel Philox actions",
         n=64, T=2000, mode=0, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 2000,
@@ -153,6 +162,10 @@ def oracle_sample(w):
     import oracle
     from paper_2603_12145_b200.inputs import explicit_actions
     n_sample = min(w["n"], 256 if w["obs_mode"] == 1 else 8192)
+    if w.get("env") == "cartpole":
+        from oracle import cartpole as oracle_cartpole
+        o = oracle_cartpole.OracleCartPole(n_sample, SEED)
+        return o, n_sample, (lambda: o.rollout(w["T"], w["mode"]))
     o = oracle.OraclePong(n_sample, SEED, obs_mode=w["obs_mode"], frameskip=w["frameskip"])
     if w["mode"] == 2:
         acts = explicit_actions(w["T"], n_sample, seed=SEED)
@@ -249,16 +262,28 @@ def main():
     warmup = max(args.warmup, 3)
     # default launch count: about 0.3 s of timed work
     default_steps = {"rollout65k": 5000, "rollout1m": 1500, "pixels16k": 200, "step4096": 20000,
+                     "cartpole65k": 5000, "cartpole1m": 1500,
                      "small64": 300}[args.workload]
     steps = args.steps if args.steps > 0 else default_steps
 
     env_id_base, _ = sharding.shard(rank, world, N)
-    env = pong.PongEnv(N, SEED, obs_mode=w["obs_mode"], frameskip=w["frameskip"],
-                       env_id_base=env_id_base)
-    obs = env.ring if pixels else torch.empty((T, N, 6), dtype=torch.float32, device="cuda")
+    is_cartpole = w.get("env") == "cartpole"
+    obs_width = 4 if is_cartpole else 6
+    if is_cartpole:
+        from paper_2603_12145_b200 import cartpole
+        cartpole.load()
+        env = cartpole.CartPoleEnv(N, SEED, env_id_base=env_id_base)
+        rollout_host = cartpole.cartpole_rollout_host
+    else:
+        env = pong.PongEnv(N, SEED, obs_mode=w["obs_mode"], frameskip=w["frameskip"],
+                           env_id_base=env_id_base)
+        rollout_host = pong.pong_rollout_host
+    obs = env.ring if pixels else torch.empty((T, N, obs_width), dtype=torch.float32, device="cuda")
     reward = torch.empty((T, N), dtype=torch.float32, device="cuda")
     done = torch.empty((T, N), dtype=torch.uint8, device="cuda")
     acts_np = explicit_actions(T, N, seed=SEED)
+    if is_cartpole:
+        acts_np = acts_np & 1
     acts_d = torch.from_numpy(acts_np).cuda() if mode == 2 else None
     l2_note = ("each step writes %.0f MB of outputs, larger than the 126 MB L2; no flush"
                % (env_steps_per_launch * w["bytes"] / 1e6))
@@ -352,16 +377,16 @@ def main():
     e2e_steps = max(args.e2e_steps, 1)
     acts_h = torch.from_numpy(acts_np).pin_memory()
     obs_h = (torch.zeros((N, 4, 84, 84), dtype=torch.uint8) if pixels
-             else torch.empty((T, N, 6), dtype=torch.float32)).pin_memory()
+             else torch.empty((T, N, obs_width), dtype=torch.float32)).pin_memory()
     rew_h = torch.empty((T, N), dtype=torch.float32).pin_memory()
     done_h = torch.empty((T, N), dtype=torch.uint8).pin_memory()
     env._stream()
     for _ in range(2):
-        pong.pong_rollout_host(env.h, T, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
+        rollout_host(env.h, T, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
     barrier()
     e0 = time.perf_counter()
     for _ in range(e2e_steps):
-        pong.pong_rollout_host(env.h, T, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
+        rollout_host(env.h, T, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - e0
     e2e_s = sharding.max_over_ranks(e2e_s, device="cuda")
@@ -381,7 +406,8 @@ def main():
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
             "warmup": warmup, "ms_per_step": kernel_ms, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "int32", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32" if is_cartpole else "int32",
+            "data": "synthetic",
             "config": {
                 "workload": w["name"], "workload_key": args.workload, "n_envs_per_gpu": N, "T": T,
                 "frameskip": w["frameskip"], "seed": SEED, "env_steps_per_step": env_steps_per_launch,
@@ -403,7 +429,8 @@ def main():
             "gpu_launches": int(launches),
             "clocks": sampler.summary(w0, w1),
             "segments": {"n": n_seg, "mean": mean, "std": std, "cv": std / mean},
-            "episode_stats": {"episodes": stats[0], "sum_return": stats[1], "sum_length": stats[2]},
+            "episode_stats": ({"episodes": stats[0], "sum_length": stats[1]} if is_cartpole else
+                              {"episodes": stats[0], "sum_return": stats[1], "sum_length": stats[2]}),
         }
         if graph_info is not None:
             line["cuda_graph"] = graph_info

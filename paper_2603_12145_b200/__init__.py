@@ -4,4 +4,4 @@
 include/pong.h; `paper_2603_12145_b200.build` compiles it; `inputs` holds the
 seeded synthetic input generators.  Importing the package loads nothing.
 """
-__all__ = ["pong", "build", "inputs", "sharding", "verify"]
+__all__ = ["pong", "cartpole", "build", "inputs", "sharding", "verify"]

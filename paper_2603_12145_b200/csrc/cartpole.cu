@@ -1,0 +1,505 @@
+// Batched CartPole for sm_100a: kernels and the C ABI declared in
+// include/cartpole.h.  One thread per env; the rollout kernel keeps the state
+// in registers across T steps and streams obs (one coalesced 16-byte store per
+// env-step), reward and done to HBM.  All arithmetic is binary32 with explicit
+// round-to-nearest intrinsics so that the compiler cannot fuse a multiply with an
+// add: the results are defined bit for bit by the order written in the header.
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include <cuda_runtime.h>
+
+#include "../../include/cartpole.h"
+
+namespace cartpole {
+
+constexpr uint32_t kM0 = 0xD2511F53u, kM1 = 0xCD9E8D57u, kW0 = 0x9E3779B9u, kW1 = 0xBB67AE85u;
+constexpr int kMaxSteps = 500;
+
+struct RoundKeys {
+    uint32_t k[20];
+};
+
+struct Args {
+    float4 *plane_f;         // [n] x, xd, th, thd
+    int2 *plane_i;           // [n] steps, episode
+    long long *stats;        // [2] episodes, sum of lengths
+    const uint8_t *actions;  // explicit mode
+    float4 *obs;             // [T][n]
+    float *reward;           // [T][n]
+    uint8_t *done;           // [T][n]
+    RoundKeys rk;
+    unsigned long long t0;
+    uint32_t env_id_base;
+    int n, T, action_mode, const_action;
+};
+
+__device__ __forceinline__ void philox(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                       const RoundKeys &rk, uint32_t (&out)[4])
+{
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint64_t p0 = (uint64_t)kM0 * c0;
+        const uint64_t p1 = (uint64_t)kM1 * c2;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk.k[2 * r];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk.k[2 * r + 1];
+        c1 = (uint32_t)p1;
+        c3 = (uint32_t)p0;
+        c0 = n0;
+        c2 = n2;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+struct Env {
+    float x, xd, th, thd;
+    int steps, episode;
+};
+
+__device__ __forceinline__ float start_value(uint32_t word)
+{
+    float f = __uint2float_rn(word >> 8);            // 24 bits, exact
+    f = __fmul_rn(f, 5.9604644775390625e-08f);       // 2^-24, exact
+    f = __fsub_rn(f, 0.5f);                          // exact
+    return __fmul_rn(f, 0.1f);
+}
+
+__device__ __forceinline__ void reset_env(Env &e, uint32_t env_id, uint32_t episode, const RoundKeys &rk)
+{
+    uint32_t o[4];
+    philox(0u, episode, env_id, 2u, rk, o);
+    e.x = start_value(o[0]);
+    e.xd = start_value(o[1]);
+    e.th = start_value(o[2]);
+    e.thd = start_value(o[3]);
+    e.steps = 0;
+    e.episode = (int)episode;
+}
+
+// One step; returns done.  On done the env is reset and the episode counted.
+__device__ __forceinline__ bool step_env(Env &e, int action, uint32_t env_id, const RoundKeys &rk,
+                                         int &episodes, int &sum_length)
+{
+    const float force = action ? 10.0f : -10.0f;
+    const float z = __fmul_rn(e.th, e.th);
+    float p = 1.0f / 362880.0f;
+    p = __fadd_rn(__fmul_rn(p, z), -1.0f / 5040.0f);
+    p = __fadd_rn(__fmul_rn(p, z), 1.0f / 120.0f);
+    p = __fadd_rn(__fmul_rn(p, z), -1.0f / 6.0f);
+    p = __fadd_rn(__fmul_rn(p, z), 1.0f);
+    const float s = __fmul_rn(e.th, p);
+    float q = 1.0f / 40320.0f;
+    q = __fadd_rn(__fmul_rn(q, z), -1.0f / 720.0f);
+    q = __fadd_rn(__fmul_rn(q, z), 1.0f / 24.0f);
+    q = __fadd_rn(__fmul_rn(q, z), -0.5f);
+    const float c = __fadd_rn(__fmul_rn(q, z), 1.0f);
+
+    const float t3 = __fmul_rn(__fmul_rn(0.05f, __fmul_rn(e.thd, e.thd)), s);
+    const float temp = __fdiv_rn(__fadd_rn(force, t3), 1.1f);
+    const float num = __fsub_rn(__fmul_rn(9.8f, s), __fmul_rn(c, temp));
+    const float d2 = __fdiv_rn(__fmul_rn(0.1f, __fmul_rn(c, c)), 1.1f);
+    const float den = __fmul_rn(0.5f, __fsub_rn(4.0f / 3.0f, d2));
+    const float thetaacc = __fdiv_rn(num, den);
+    const float m3 = __fdiv_rn(__fmul_rn(__fmul_rn(0.05f, thetaacc), c), 1.1f);
+    const float xacc = __fsub_rn(temp, m3);
+
+    const float dx = __fmul_rn(0.02f, e.xd);
+    const float dxd = __fmul_rn(0.02f, xacc);
+    const float dth = __fmul_rn(0.02f, e.thd);
+    const float dthd = __fmul_rn(0.02f, thetaacc);
+    e.x = __fadd_rn(e.x, dx);
+    e.xd = __fadd_rn(e.xd, dxd);
+    e.th = __fadd_rn(e.th, dth);
+    e.thd = __fadd_rn(e.thd, dthd);
+    e.steps += 1;
+
+    const float th_limit = 0.20943951023931953f;
+    const bool done = e.x < -2.4f || e.x > 2.4f || e.th < -th_limit || e.th > th_limit ||
+                      e.steps >= kMaxSteps;
+    if (done) {
+        episodes += 1;
+        sum_length += e.steps;
+        reset_env(e, env_id, (uint32_t)e.episode + 1u, rk);
+    }
+    return done;
+}
+
+__device__ __forceinline__ void flush_stats(int episodes, int sum_length, long long *stats)
+{
+    const int ep = __reduce_add_sync(0xffffffffu, episodes);
+    if (ep == 0) return;
+    const int ls = __reduce_add_sync(0xffffffffu, sum_length);
+    if ((threadIdx.x & 31) == 0) {
+        atomicAdd(reinterpret_cast<unsigned long long *>(stats + 0), (unsigned long long)(long long)ep);
+        atomicAdd(reinterpret_cast<unsigned long long *>(stats + 1), (unsigned long long)(long long)ls);
+    }
+}
+
+constexpr int kBlock = 128;
+
+__global__ void __launch_bounds__(kBlock) k_cartpole_reset(const __grid_constant__ Args a)
+{
+    const int n = blockIdx.x * kBlock + threadIdx.x;
+    if (n >= a.n) return;
+    Env e;
+    reset_env(e, a.env_id_base + (uint32_t)n, 0u, a.rk);
+    a.plane_f[n] = make_float4(e.x, e.xd, e.th, e.thd);
+    a.plane_i[n] = make_int2(e.steps, e.episode);
+    if (a.obs != nullptr) a.obs[n] = make_float4(e.x, e.xd, e.th, e.thd);
+}
+
+// MODE 0: Philox actions (one block of four words serves four steps), 2: explicit
+// bytes, 3: constant.
+template <int MODE>
+__global__ void __launch_bounds__(kBlock) k_cartpole_rollout(const __grid_constant__ Args a)
+{
+    const int n = blockIdx.x * kBlock + threadIdx.x;
+    int episodes = 0, sum_length = 0;
+    if (n < a.n) {
+        Env e;
+        {
+            const float4 f = a.plane_f[n];
+            const int2 i = a.plane_i[n];
+            e.x = f.x; e.xd = f.y; e.th = f.z; e.thd = f.w;
+            e.steps = i.x; e.episode = i.y;
+        }
+        const uint32_t env_id = a.env_id_base + (uint32_t)n;
+        const size_t stride = (size_t)a.n;
+        float4 *obs = a.obs + n;
+        float *rew = a.reward + n;
+        uint8_t *dn = a.done + n;
+        const uint8_t *act = MODE == 2 ? a.actions + n : nullptr;
+        const unsigned long long t_end = a.t0 + (unsigned long long)a.T;
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        for (unsigned long long tt = a.t0; tt < t_end; ++tt) {
+            int action;
+            if (MODE == 0) {
+                if (tt == a.t0 || (tt & 3ull) == 0)
+                    philox((uint32_t)(tt >> 2), env_id, (uint32_t)(tt >> 34), 3u, a.rk, w);
+                const int sel = (int)(tt & 3ull);
+                const uint32_t word = sel == 0 ? w[0] : sel == 1 ? w[1] : sel == 2 ? w[2] : w[3];
+                action = (int)(word & 1u);
+            } else if (MODE == 2) {
+                action = *act & 1u;
+                act += stride;
+            } else {
+                action = a.const_action;
+            }
+            const bool done = step_env(e, action, env_id, a.rk, episodes, sum_length);
+            *obs = make_float4(e.x, e.xd, e.th, e.thd);
+            *rew = 1.0f;
+            *dn = done ? 1 : 0;
+            obs += stride;
+            rew += stride;
+            dn += stride;
+        }
+        a.plane_f[n] = make_float4(e.x, e.xd, e.th, e.thd);
+        a.plane_i[n] = make_int2(e.steps, e.episode);
+    }
+    flush_stats(episodes, sum_length, a.stats);
+}
+
+}  // namespace cartpole
+
+// ---- C ABI ----------------------------------------------------------------------------
+
+struct cartpole_env {
+    int n = 0;
+    uint64_t seed = 0;
+    int env_id_base = 0;
+    cudaStream_t stream = nullptr;
+    void *block = nullptr;
+    float4 *plane_f = nullptr;
+    int2 *plane_i = nullptr;
+    long long *stats = nullptr;
+    uint64_t t = 0;
+    int64_t launches = 0;
+    cartpole::RoundKeys rk;
+    void *stage = nullptr;
+    size_t stage_bytes = 0;
+};
+
+namespace {
+
+cartpole::Args base_args(const cartpole_env *h)
+{
+    cartpole::Args a;
+    std::memset(&a, 0, sizeof(a));
+    a.plane_f = h->plane_f;
+    a.plane_i = h->plane_i;
+    a.stats = h->stats;
+    a.rk = h->rk;
+    a.t0 = h->t;
+    a.env_id_base = (uint32_t)h->env_id_base;
+    a.n = h->n;
+    a.T = 1;
+    return a;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int do_reset(cartpole_env *h, float *obs_out)
+{
+    if (obs_out != nullptr && !aligned16(obs_out)) return CARTPOLE_EALIGN;
+    if (cudaMemsetAsync(h->stats, 0, 2 * sizeof(long long), h->stream) != cudaSuccess) return CARTPOLE_ECUDA;
+    h->t = 0;
+    cartpole::Args a = base_args(h);
+    a.obs = reinterpret_cast<float4 *>(obs_out);
+    cartpole::k_cartpole_reset<<<(h->n + cartpole::kBlock - 1) / cartpole::kBlock, cartpole::kBlock, 0, h->stream>>>(a);
+    h->launches += 1;
+    return cudaGetLastError() == cudaSuccess ? CARTPOLE_OK : CARTPOLE_ECUDA;
+}
+
+int check_args(const cartpole_env *h, int T, int mode, const uint8_t *actions, const void *obs,
+               const void *reward, const void *done, int *const_action)
+{
+    if (h == nullptr) return CARTPOLE_ENULL;
+    if (T < 1 || (uint64_t)T * (uint64_t)h->n > (1ull << 40)) return CARTPOLE_EINVAL;
+    if (mode != CARTPOLE_ACT_PHILOX && mode != CARTPOLE_ACT_EXPLICIT && mode != CARTPOLE_ACT_CONSTANT)
+        return CARTPOLE_EMODE;
+    if (obs == nullptr || reward == nullptr || done == nullptr) return CARTPOLE_ENULL;
+    if (mode != CARTPOLE_ACT_PHILOX && actions == nullptr) return CARTPOLE_ENULL;
+    *const_action = 0;
+    if (mode == CARTPOLE_ACT_CONSTANT) {
+        if (actions[0] > 1) return CARTPOLE_EINVAL;
+        *const_action = actions[0];
+    }
+    return CARTPOLE_OK;
+}
+
+int do_rollout(cartpole_env *h, int T, int mode, const uint8_t *actions, int const_action, float *obs,
+               float *reward, uint8_t *done)
+{
+    cartpole::Args a = base_args(h);
+    a.T = T;
+    a.action_mode = mode;
+    a.actions = actions;
+    a.const_action = const_action;
+    a.obs = reinterpret_cast<float4 *>(obs);
+    a.reward = reward;
+    a.done = done;
+    const int grid = (h->n + cartpole::kBlock - 1) / cartpole::kBlock;
+    if (mode == CARTPOLE_ACT_PHILOX)
+        cartpole::k_cartpole_rollout<0><<<grid, cartpole::kBlock, 0, h->stream>>>(a);
+    else if (mode == CARTPOLE_ACT_EXPLICIT)
+        cartpole::k_cartpole_rollout<2><<<grid, cartpole::kBlock, 0, h->stream>>>(a);
+    else
+        cartpole::k_cartpole_rollout<3><<<grid, cartpole::kBlock, 0, h->stream>>>(a);
+    if (cudaGetLastError() != cudaSuccess) return CARTPOLE_ECUDA;
+    h->launches += 1;
+    h->t += (uint64_t)T;
+    return CARTPOLE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int cartpole_create(cartpole_env **out, int n_envs, uint64_t seed, int env_id_base)
+{
+    if (out == nullptr) return CARTPOLE_ENULL;
+    *out = nullptr;
+    if (n_envs < 1 || env_id_base < 0 || (int64_t)env_id_base + n_envs > 0x7fffffffLL) return CARTPOLE_EINVAL;
+    cartpole_env *h = new (std::nothrow) cartpole_env();
+    if (h == nullptr) return CARTPOLE_ENOMEM;
+    h->n = n_envs;
+    h->seed = seed;
+    h->env_id_base = env_id_base;
+    for (int r = 0; r < 10; ++r) {
+        h->rk.k[2 * r] = (uint32_t)seed + (uint32_t)r * cartpole::kW0;
+        h->rk.k[2 * r + 1] = (uint32_t)(seed >> 32) + (uint32_t)r * cartpole::kW1;
+    }
+    const size_t n = (size_t)n_envs;
+    const cudaError_t err = cudaMalloc(&h->block, n * (sizeof(float4) + sizeof(int2)) + 64);
+    if (err != cudaSuccess) {
+        cudaGetLastError();
+        delete h;
+        return err == cudaErrorMemoryAllocation ? CARTPOLE_ENOMEM : CARTPOLE_ECUDA;
+    }
+    h->plane_f = static_cast<float4 *>(h->block);
+    h->plane_i = reinterpret_cast<int2 *>(h->plane_f + n);
+    h->stats = reinterpret_cast<long long *>(h->plane_i + n);
+    const int rc = do_reset(h, nullptr);
+    if (rc != CARTPOLE_OK) {
+        cudaFree(h->block);
+        delete h;
+        return rc;
+    }
+    *out = h;
+    return CARTPOLE_OK;
+}
+
+int cartpole_destroy(cartpole_env *h)
+{
+    if (h == nullptr) return CARTPOLE_OK;
+    int rc = CARTPOLE_OK;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) rc = CARTPOLE_ECUDA;
+    if (h->stage != nullptr && cudaFree(h->stage) != cudaSuccess) rc = CARTPOLE_ECUDA;
+    if (cudaFree(h->block) != cudaSuccess) rc = CARTPOLE_ECUDA;
+    delete h;
+    return rc;
+}
+
+int cartpole_set_stream(cartpole_env *h, void *cuda_stream)
+{
+    if (h == nullptr) return CARTPOLE_ENULL;
+    h->stream = static_cast<cudaStream_t>(cuda_stream);
+    return CARTPOLE_OK;
+}
+
+int cartpole_reset(cartpole_env *h, float *obs_out)
+{
+    if (h == nullptr) return CARTPOLE_ENULL;
+    return do_reset(h, obs_out);
+}
+
+int cartpole_step(cartpole_env *h, const uint8_t *actions, float *obs, float *reward, uint8_t *done)
+{
+    if (h == nullptr || actions == nullptr || obs == nullptr || reward == nullptr || done == nullptr)
+        return CARTPOLE_ENULL;
+    if (!aligned16(obs)) return CARTPOLE_EALIGN;
+    return do_rollout(h, 1, CARTPOLE_ACT_EXPLICIT, actions, 0, obs, reward, done);
+}
+
+int cartpole_rollout(cartpole_env *h, int T, int action_mode, const uint8_t *actions, float *obs,
+                     float *reward, uint8_t *done)
+{
+    int const_action = 0;
+    const int rc = check_args(h, T, action_mode, actions, obs, reward, done, &const_action);
+    if (rc != CARTPOLE_OK) return rc;
+    if (!aligned16(obs)) return CARTPOLE_EALIGN;
+    return do_rollout(h, T, action_mode, actions, const_action, obs, reward, done);
+}
+
+int cartpole_rollout_host(cartpole_env *h, int T, int action_mode, const uint8_t *actions_host,
+                          float *obs_host, float *reward_host, uint8_t *done_host)
+{
+    int const_action = 0;
+    const int rc = check_args(h, T, action_mode, actions_host, obs_host, reward_host, done_host, &const_action);
+    if (rc != CARTPOLE_OK) return rc;
+    const size_t tn = (size_t)T * (size_t)h->n;
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    const size_t off_reward = up(tn * 16), off_done = off_reward + up(tn * 4), off_act = off_done + up(tn);
+    const size_t need = off_act + up(action_mode == CARTPOLE_ACT_EXPLICIT ? tn : 0);
+    if (need > h->stage_bytes) {
+        if (cudaStreamSynchronize(h->stream) != cudaSuccess) return CARTPOLE_ECUDA;
+        if (h->stage != nullptr) cudaFree(h->stage);
+        h->stage = nullptr;
+        h->stage_bytes = 0;
+        if (cudaMalloc(&h->stage, need) != cudaSuccess) {
+            cudaGetLastError();
+            return CARTPOLE_ENOMEM;
+        }
+        h->stage_bytes = need;
+    }
+    char *base = static_cast<char *>(h->stage);
+    float *d_obs = reinterpret_cast<float *>(base);
+    float *d_reward = reinterpret_cast<float *>(base + off_reward);
+    uint8_t *d_done = reinterpret_cast<uint8_t *>(base + off_done);
+    uint8_t *d_act = reinterpret_cast<uint8_t *>(base + off_act);
+    const uint8_t *actions = actions_host;
+    if (action_mode == CARTPOLE_ACT_EXPLICIT) {
+        if (cudaMemcpyAsync(d_act, actions_host, tn, cudaMemcpyHostToDevice, h->stream) != cudaSuccess)
+            return CARTPOLE_ECUDA;
+        actions = d_act;
+    }
+    const int rr = do_rollout(h, T, action_mode, actions, const_action, d_obs, d_reward, d_done);
+    if (rr != CARTPOLE_OK) return rr;
+    if (cudaMemcpyAsync(obs_host, d_obs, tn * 16, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+        cudaMemcpyAsync(reward_host, d_reward, tn * 4, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+        cudaMemcpyAsync(done_host, d_done, tn, cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+        cudaStreamSynchronize(h->stream) != cudaSuccess)
+        return CARTPOLE_ECUDA;
+    return CARTPOLE_OK;
+}
+
+int cartpole_episode_stats(cartpole_env *h, int64_t *episodes, int64_t *sum_length, int clear)
+{
+    if (h == nullptr) return CARTPOLE_ENULL;
+    long long v[2] = {0, 0};
+    if (cudaMemcpyAsync(v, h->stats, sizeof(v), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess)
+        return CARTPOLE_ECUDA;
+    if (clear && cudaMemsetAsync(h->stats, 0, sizeof(v), h->stream) != cudaSuccess) return CARTPOLE_ECUDA;
+    if (cudaStreamSynchronize(h->stream) != cudaSuccess) return CARTPOLE_ECUDA;
+    if (episodes) *episodes = v[0];
+    if (sum_length) *sum_length = v[1];
+    return CARTPOLE_OK;
+}
+
+int cartpole_get_state(cartpole_env *h, float *host_f, int32_t *host_i, uint64_t *t)
+{
+    if (h == nullptr || host_f == nullptr || host_i == nullptr) return CARTPOLE_ENULL;
+    const size_t n = (size_t)h->n;
+    std::vector<float4> f;
+    std::vector<int2> i;
+    try {
+        f.resize(n);
+        i.resize(n);
+    } catch (...) {
+        return CARTPOLE_ENOMEM;
+    }
+    if (cudaMemcpyAsync(f.data(), h->plane_f, n * sizeof(float4), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+        cudaMemcpyAsync(i.data(), h->plane_i, n * sizeof(int2), cudaMemcpyDeviceToHost, h->stream) != cudaSuccess ||
+        cudaStreamSynchronize(h->stream) != cudaSuccess)
+        return CARTPOLE_ECUDA;
+    for (size_t k = 0; k < n; ++k) {
+        host_f[0 * n + k] = f[k].x;
+        host_f[1 * n + k] = f[k].y;
+        host_f[2 * n + k] = f[k].z;
+        host_f[3 * n + k] = f[k].w;
+        host_i[0 * n + k] = i[k].x;
+        host_i[1 * n + k] = i[k].y;
+    }
+    if (t) *t = h->t;
+    return CARTPOLE_OK;
+}
+
+int cartpole_set_state(cartpole_env *h, const float *host_f, const int32_t *host_i, uint64_t t)
+{
+    if (h == nullptr || host_f == nullptr || host_i == nullptr) return CARTPOLE_ENULL;
+    const size_t n = (size_t)h->n;
+    std::vector<float4> f;
+    std::vector<int2> i;
+    try {
+        f.resize(n);
+        i.resize(n);
+    } catch (...) {
+        return CARTPOLE_ENOMEM;
+    }
+    for (size_t k = 0; k < n; ++k) {
+        f[k] = make_float4(host_f[k], host_f[n + k], host_f[2 * n + k], host_f[3 * n + k]);
+        i[k] = make_int2(host_i[k], host_i[n + k]);
+        if (!std::isfinite(f[k].x) || !std::isfinite(f[k].y) || !std::isfinite(f[k].z) ||
+            !std::isfinite(f[k].w) || i[k].x < 0 || i[k].x >= cartpole::kMaxSteps || i[k].y < 0)
+            return CARTPOLE_EINVAL;
+    }
+    if (cudaMemcpyAsync(h->plane_f, f.data(), n * sizeof(float4), cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+        cudaMemcpyAsync(h->plane_i, i.data(), n * sizeof(int2), cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+        cudaStreamSynchronize(h->stream) != cudaSuccess)
+        return CARTPOLE_ECUDA;
+    h->t = t;
+    return CARTPOLE_OK;
+}
+
+int cartpole_num_envs(const cartpole_env *h) { return h ? h->n : CARTPOLE_ENULL; }
+
+int64_t cartpole_launch_count(const cartpole_env *h) { return h ? h->launches : (int64_t)CARTPOLE_ENULL; }
+
+const char *cartpole_strerror(int code)
+{
+    switch (code) {
+    case CARTPOLE_OK: return "ok";
+    case CARTPOLE_EINVAL: return "invalid argument (size, T, action or state value)";
+    case CARTPOLE_ENULL: return "required pointer is NULL";
+    case CARTPOLE_EALIGN: return "obs pointer is not 16-byte aligned";
+    case CARTPOLE_ECUDA: return "a CUDA runtime call or kernel launch failed";
+    case CARTPOLE_EMODE: return "unknown action_mode";
+    case CARTPOLE_ENOMEM: return "out of host or device memory";
+    default: return "unknown error code";
+    }
+}
+
+}  // extern "C"

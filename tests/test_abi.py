@@ -11,10 +11,10 @@ from paper_2603_12145_b200 import build, pong
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def declared_symbols():
-    text = open(os.path.join(ROOT, "include", "pong.h")).read()
+def declared_symbols(header="pong.h", prefix="pong"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(pong_[a-z_]+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(%s_[a-z_]+)\s*\(" % prefix, text)))
 
 
 def test_library_builds_and_exports_every_declared_symbol():
@@ -63,3 +63,20 @@ def test_no_cpu_fallback_without_device():
     with pytest.raises(pong.PongError) as ei:
         pong.pong_create(4, 0)
     assert ei.value.code == -4
+
+
+def test_cartpole_library_exports_every_declared_symbol():
+    from paper_2603_12145_b200 import cartpole
+    lib = ctypes.CDLL(build.build_one("libcartpole_b200.so"))
+    names = declared_symbols("cartpole.h", "cartpole")
+    assert len(names) >= 13
+    for name in names:
+        assert hasattr(lib, name), name
+    assert set(names) == set(cartpole.EXPORTS)
+    L = cartpole.load(build_if_missing=True)
+    assert cartpole.strerror(0) == "ok" and cartpole.strerror(-99) == "unknown error code"
+    assert L.cartpole_reset(None, None) == -2 and L.cartpole_destroy(None) == 0
+    h = ctypes.c_void_p()
+    assert L.cartpole_create(ctypes.byref(h), 0, 0, 0) == -1
+    assert L.cartpole_create(ctypes.byref(h), 4, 0, -1) == -1
+    assert L.cartpole_create(None, 4, 0, 0) == -2
