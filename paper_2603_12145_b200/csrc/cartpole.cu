@@ -79,9 +79,8 @@ __device__ __forceinline__ void reset_env(Env &e, uint32_t env_id, uint32_t epis
     e.episode = (int)episode;
 }
 
-// One step; returns done.  On done the env is reset and the episode counted.
-__device__ __forceinline__ bool step_env(Env &e, int action, uint32_t env_id, const RoundKeys &rk,
-                                         int &episodes, int &sum_length)
+// The dynamics of one step (no termination handling).
+__device__ __forceinline__ void advance(Env &e, int action)
 {
     const float force = action ? 10.0f : -10.0f;
     const float z = __fmul_rn(e.th, e.th);
@@ -98,12 +97,13 @@ __device__ __forceinline__ bool step_env(Env &e, int action, uint32_t env_id, co
     const float c = __fadd_rn(__fmul_rn(q, z), 1.0f);
 
     const float t3 = __fmul_rn(__fmul_rn(0.05f, __fmul_rn(e.thd, e.thd)), s);
-    const float temp = __fdiv_rn(__fadd_rn(force, t3), 1.1f);
+    const float inv_total = 1.0f / 1.1f;  // reciprocal of the total mass, rounded once
+    const float temp = __fmul_rn(__fadd_rn(force, t3), inv_total);
     const float num = __fsub_rn(__fmul_rn(9.8f, s), __fmul_rn(c, temp));
-    const float d2 = __fdiv_rn(__fmul_rn(0.1f, __fmul_rn(c, c)), 1.1f);
+    const float d2 = __fmul_rn(__fmul_rn(0.1f, __fmul_rn(c, c)), inv_total);
     const float den = __fmul_rn(0.5f, __fsub_rn(4.0f / 3.0f, d2));
     const float thetaacc = __fdiv_rn(num, den);
-    const float m3 = __fdiv_rn(__fmul_rn(__fmul_rn(0.05f, thetaacc), c), 1.1f);
+    const float m3 = __fmul_rn(__fmul_rn(__fmul_rn(0.05f, thetaacc), c), inv_total);
     const float xacc = __fsub_rn(temp, m3);
 
     const float dx = __fmul_rn(0.02f, e.xd);
@@ -115,16 +115,12 @@ __device__ __forceinline__ bool step_env(Env &e, int action, uint32_t env_id, co
     e.th = __fadd_rn(e.th, dth);
     e.thd = __fadd_rn(e.thd, dthd);
     e.steps += 1;
+}
 
+__device__ __forceinline__ bool terminated(const Env &e)
+{
     const float th_limit = 0.20943951023931953f;
-    const bool done = e.x < -2.4f || e.x > 2.4f || e.th < -th_limit || e.th > th_limit ||
-                      e.steps >= kMaxSteps;
-    if (done) {
-        episodes += 1;
-        sum_length += e.steps;
-        reset_env(e, env_id, (uint32_t)e.episode + 1u, rk);
-    }
-    return done;
+    return e.x < -2.4f || e.x > 2.4f || e.th < -th_limit || e.th > th_limit || e.steps >= kMaxSteps;
 }
 
 __device__ __forceinline__ void flush_stats(int episodes, int sum_length, long long *stats)
@@ -151,12 +147,26 @@ __global__ void __launch_bounds__(kBlock) k_cartpole_reset(const __grid_constant
     if (a.obs != nullptr) a.obs[n] = make_float4(e.x, e.xd, e.th, e.thd);
 }
 
+// Start states of coming episodes.  A random policy ends an episode about every 22
+// steps, so in nearly every step some lane of a warp needs a reset; computing its
+// Philox block there would run ten rounds for one or two live lanes.  Instead every
+// thread fills, with all lanes busy, a private column of this table with the start
+// states of its next episodes before each chunk of steps and pops one per episode
+// end.  An episode that starts from a reset cannot end before its 8th step (the
+// pole needs that long to reach 12 degrees from |th|, |thd| <= 0.05), so a chunk of
+// S steps ends at most 1 + (S-1)/8 episodes; should a column still run out, the
+// start state is computed in place.
+constexpr int kChunk = 128;
+constexpr int kTable = 1 + (kChunk - 1) / 8;
+
 // MODE 0: Philox actions (one block of four words serves four steps), 2: explicit
-// bytes, 3: constant.
-template <int MODE>
+// bytes, 3: constant.  FULL: t0 and T are multiples of 4.
+template <int MODE, bool FULL>
 __global__ void __launch_bounds__(kBlock) k_cartpole_rollout(const __grid_constant__ Args a)
 {
-    const int n = blockIdx.x * kBlock + threadIdx.x;
+    __shared__ float4 table[kTable][kBlock];
+    const int tid = threadIdx.x;
+    const int n = blockIdx.x * kBlock + tid;
     int episodes = 0, sum_length = 0;
     if (n < a.n) {
         Env e;
@@ -173,28 +183,51 @@ __global__ void __launch_bounds__(kBlock) k_cartpole_rollout(const __grid_consta
         uint8_t *dn = a.done + n;
         const uint8_t *act = MODE == 2 ? a.actions + n : nullptr;
         const unsigned long long t_end = a.t0 + (unsigned long long)a.T;
-        uint32_t w[4] = {0u, 0u, 0u, 0u};
-        for (unsigned long long tt = a.t0; tt < t_end; ++tt) {
-            int action;
-            if (MODE == 0) {
-                if (tt == a.t0 || (tt & 3ull) == 0)
-                    philox((uint32_t)(tt >> 2), env_id, (uint32_t)(tt >> 34), 3u, a.rk, w);
-                const int sel = (int)(tt & 3ull);
-                const uint32_t word = sel == 0 ? w[0] : sel == 1 ? w[1] : sel == 2 ? w[2] : w[3];
-                action = (int)(word & 1u);
-            } else if (MODE == 2) {
-                action = *act & 1u;
-                act += stride;
-            } else {
-                action = a.const_action;
+
+        for (unsigned long long c0 = a.t0; c0 < t_end; c0 += kChunk) {
+            const unsigned long long c1 = c0 + kChunk < t_end ? c0 + kChunk : t_end;
+            const int filled = 1 + ((int)(c1 - c0) - 1) / 8;
+            for (int k = 0; k < filled; ++k) {
+                Env r;
+                reset_env(r, env_id, (uint32_t)(e.episode + 1 + k), a.rk);
+                table[k][tid] = make_float4(r.x, r.xd, r.th, r.thd);
             }
-            const bool done = step_env(e, action, env_id, a.rk, episodes, sum_length);
-            *obs = make_float4(e.x, e.xd, e.th, e.thd);
-            *rew = 1.0f;
-            *dn = done ? 1 : 0;
-            obs += stride;
-            rew += stride;
-            dn += stride;
+            int used = 0;
+            for (unsigned long long g = c0 >> 2; g <= (c1 - 1) >> 2; ++g) {
+                uint32_t w[4] = {0u, 0u, 0u, 0u};
+                if (MODE == 0) philox((uint32_t)g, env_id, (uint32_t)(g >> 32), 3u, a.rk, w);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const unsigned long long tt = g * 4 + j;
+                    if (FULL || (tt >= c0 && tt < c1)) {
+                        int action;
+                        if (MODE == 0) action = (int)(w[j] & 1u);
+                        else if (MODE == 2) { action = *act & 1u; act += stride; }
+                        else action = a.const_action;
+                        advance(e, action);
+                        const bool done = terminated(e);
+                        if (done) {
+                            episodes += 1;
+                            sum_length += e.steps;
+                            e.episode += 1;
+                            e.steps = 0;
+                            if (used < filled) {
+                                const float4 r = table[used][tid];
+                                e.x = r.x; e.xd = r.y; e.th = r.z; e.thd = r.w;
+                                used += 1;
+                            } else {
+                                reset_env(e, env_id, (uint32_t)e.episode, a.rk);
+                            }
+                        }
+                        *obs = make_float4(e.x, e.xd, e.th, e.thd);
+                        *rew = 1.0f;
+                        *dn = done ? 1 : 0;
+                        obs += stride;
+                        rew += stride;
+                        dn += stride;
+                    }
+                }
+            }
         }
         a.plane_f[n] = make_float4(e.x, e.xd, e.th, e.thd);
         a.plane_i[n] = make_int2(e.steps, e.episode);
@@ -282,12 +315,16 @@ int do_rollout(cartpole_env *h, int T, int mode, const uint8_t *actions, int con
     a.reward = reward;
     a.done = done;
     const int grid = (h->n + cartpole::kBlock - 1) / cartpole::kBlock;
-    if (mode == CARTPOLE_ACT_PHILOX)
-        cartpole::k_cartpole_rollout<0><<<grid, cartpole::kBlock, 0, h->stream>>>(a);
-    else if (mode == CARTPOLE_ACT_EXPLICIT)
-        cartpole::k_cartpole_rollout<2><<<grid, cartpole::kBlock, 0, h->stream>>>(a);
-    else
-        cartpole::k_cartpole_rollout<3><<<grid, cartpole::kBlock, 0, h->stream>>>(a);
+    const bool full = h->t % 4 == 0 && T % 4 == 0;
+#define CARTPOLE_LAUNCH(M)                                                                       \
+    do {                                                                                         \
+        if (full) cartpole::k_cartpole_rollout<M, true><<<grid, cartpole::kBlock, 0, h->stream>>>(a);  \
+        else cartpole::k_cartpole_rollout<M, false><<<grid, cartpole::kBlock, 0, h->stream>>>(a);      \
+    } while (0)
+    if (mode == CARTPOLE_ACT_PHILOX) CARTPOLE_LAUNCH(0);
+    else if (mode == CARTPOLE_ACT_EXPLICIT) CARTPOLE_LAUNCH(2);
+    else CARTPOLE_LAUNCH(3);
+#undef CARTPOLE_LAUNCH
     if (cudaGetLastError() != cudaSuccess) return CARTPOLE_ECUDA;
     h->launches += 1;
     h->t += (uint64_t)T;
