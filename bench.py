@@ -63,11 +63,11 @@ WORKLOADS = {
     "cartpole65k": dict(
         name="CartPole fused rollout, N=65536 envs, T=128 steps per launch, in-kernel Philox actions",
         env="cartpole", n=65536, T=128, mode=0, obs_mode=0, frameskip=1, bytes=21.0 + 48.0 / 128,
-        kernel="k_cartpole_rollout", traffic=None),
+        kernel="k_cartpole_rollout", traffic=120.3e6),
     "cartpole1m": dict(
         name="CartPole fused rollout, N=1048576 envs, T=32 steps per launch, in-kernel Philox actions",
         env="cartpole", n=1048576, T=32, mode=0, obs_mode=0, frameskip=1, bytes=21.0 + 48.0 / 32,
-        kernel="k_cartpole_rollout", traffic=None),
+        kernel="k_cartpole_rollout", traffic=695.4e6),
     "small64": dict(
         name="fused vector-obs rollout, N=64 envs, T=2000 steps per launch, in-kernel Philox actions",
         n=64, T=2000, mode=0, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 2000,
