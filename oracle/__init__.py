@@ -86,6 +86,14 @@ def lib():
             L.oracle_rollout.restype = i32
             L.oracle_fill_actions.argtypes = [i32, u64, u32, u64, i32, i32, vp]
             L.oracle_fill_actions.restype = None
+            L.oracle_expn.argtypes = [ctypes.c_float]
+            L.oracle_expn.restype = ctypes.c_float
+            L.oracle_sample_action.argtypes = [vp, u32]
+            L.oracle_sample_action.restype = i32
+            L.oracle_sample_actions.argtypes = [i32, vp, vp, vp]
+            L.oracle_sample_actions.restype = None
+            L.oracle_fill_words.argtypes = [i32, u64, u32, u64, i32, vp]
+            L.oracle_fill_words.restype = None
             L.oracle_sizeof_env.argtypes = []
             L.oracle_sizeof_env.restype = i32
             assert L.oracle_sizeof_env() == ctypes.sizeof(_Env)
@@ -119,6 +127,20 @@ def action_repeat(word):
 
 def decode_action(byte, prev_action):
     return int(lib().oracle_decode_action(byte, prev_action))
+
+
+def expn(x):
+    return float(lib().oracle_expn(float(x)))
+
+
+def sample_actions(logits, words):
+    """uint8 [n] actions drawn from softmax(logits[n, 3]) with the uniform words[n]."""
+    logits = np.ascontiguousarray(logits, dtype=np.float32).reshape(-1, 3)
+    words = np.ascontiguousarray(words, dtype=np.uint32).reshape(-1)
+    assert len(words) == len(logits)
+    out = np.zeros(len(words), dtype=np.uint8)
+    lib().oracle_sample_actions(len(words), _ptr(logits), _ptr(words), _ptr(out))
+    return out
 
 
 class Env:
@@ -233,6 +255,15 @@ class OraclePong:
         lib().oracle_fill_actions(self.n, self.seed, self.env_id_base, self.t,
                                   int(T), int(sticky), _ptr(out))
         return out
+
+    def fill_words(self, T):
+        """uint32 [T, n]: the Philox action words of the next T global steps."""
+        out = np.zeros((int(T), self.n), dtype=np.uint32)
+        lib().oracle_fill_words(self.n, self.seed, self.env_id_base, self.t, int(T), _ptr(out))
+        return out
+
+    def advance_step_counter(self, steps):
+        self.t += int(steps)
 
     def episode_stats(self, clear=False):
         s = (int(self.stats.episodes), int(self.stats.sum_return),

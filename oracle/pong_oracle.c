@@ -390,3 +390,79 @@ void oracle_fill_actions(int n, uint64_t seed, uint32_t env_id_base, uint64_t t0
 }
 
 int oracle_sizeof_env(void) { return (int)sizeof(oracle_env); }
+
+/* ---- policy interface: sampling an action from three logits ---------------- */
+/* Used when a policy network drives the env (the paper's "GRU rollout"
+ * benchmark, Table "PufferLib comparisons"): the policy emits logits, an action
+ * is drawn from softmax(logits) with one uniform number per env and step, and
+ * the env steps on it.  The draw compares floating-point numbers, so it is
+ * defined in binary32 with a fixed operation order and a fixed polynomial
+ * exponential, and the uniform number is an input (the Philox action word of
+ * that env and step), so that two implementations agree on every action.
+ *
+ *   m  = max(l0, l1, l2)
+ *   ei = expn(li - m)                       expn(x) = e^x for x <= 0, below
+ *   s  = (e0 + e1) + e2
+ *   x  = ((float)(word >> 8) * 2^-24) * s   uniform in [0, s)
+ *   a  = x < e0 ? 0 : (x < e0 + e1 ? 1 : 2)
+ *
+ * expn(x): y = x * log2(e); n = floor(y + 0.5); f = y - n in [-0.5, 0.5];
+ * 2^f = ((((((P6 f + P5) f + P4) f + P3) f + P2) f + P1) f + 1 with the Taylor
+ * coefficients Pk = ln(2)^k / k!; result = 2^f scaled by 2^n (exact), and 0
+ * when n < -126.  Relative error below 3e-7 for |x| <= 1 and below 1e-6 for
+ * |x| <= 8; for larger |x| the rounding of y dominates (4e-6 at x = -80), where the value no longer matters
+ * to a softmax. */
+float oracle_expn(float x)
+{
+    if (!(x <= 0.0f)) x = 0.0f;                 /* callers pass l - max <= 0; NaN -> 0 */
+    float y = x * 1.44269504088896340736f;
+    float t = y + 0.5f;
+    float n = (float)(int)t;                    /* truncation towards zero ... */
+    if (n > t) n = n - 1.0f;                    /* ... made a floor: n = round(y) */
+    if (n < -126.0f) return 0.0f;
+    float f = y - n;
+    float p = 1.5403530393381608e-4f;           /* ln2^6/720 */
+    p = p * f; p = p + 1.3333558146428443e-3f;  /* ln2^5/120 */
+    p = p * f; p = p + 9.6181291076284772e-3f;  /* ln2^4/24 */
+    p = p * f; p = p + 5.5504108664821580e-2f;  /* ln2^3/6 */
+    p = p * f; p = p + 2.4022650695910072e-1f;  /* ln2^2/2 */
+    p = p * f; p = p + 6.9314718055994531e-1f;  /* ln2 */
+    p = p * f; p = p + 1.0f;
+    union { uint32_t u; float f; } scale;
+    scale.u = (uint32_t)((int)n + 127) << 23;   /* 2^n, n in [-126, 0] */
+    return p * scale.f;
+}
+
+int oracle_sample_action(const float logits[3], uint32_t word)
+{
+    float m = logits[0];
+    if (logits[1] > m) m = logits[1];
+    if (logits[2] > m) m = logits[2];
+    float e0 = oracle_expn(logits[0] - m);
+    float e1 = oracle_expn(logits[1] - m);
+    float e2 = oracle_expn(logits[2] - m);
+    float e01 = e0 + e1;
+    float s = e01 + e2;
+    float u = (float)(word >> 8);
+    u = u * 5.9604644775390625e-08f;            /* 2^-24 */
+    float x = u * s;
+    if (x < e0) return 0;
+    if (x < e01) return 1;
+    return 2;
+}
+
+/* actions[n] from logits[n][3] and words[n] */
+void oracle_sample_actions(int n, const float *logits, const uint32_t *words, uint8_t *actions)
+{
+    for (int i = 0; i < n; ++i) actions[i] = (uint8_t)oracle_sample_action(logits + 3 * i, words[i]);
+}
+
+/* The Philox action words of global steps t0 .. t0+T-1: words[T][n]. */
+void oracle_fill_words(int n, uint64_t seed, uint32_t env_id_base, uint64_t t0, int T,
+                       uint32_t *words)
+{
+    for (int t = 0; t < T; ++t)
+        for (int i = 0; i < n; ++i)
+            words[(size_t)t * (size_t)n + (size_t)i] =
+                oracle_action_word(seed, env_id_base + (uint32_t)i, t0 + (uint64_t)t);
+}
