@@ -10,7 +10,7 @@ statistics reduction, i.e. 8,388,608 env-steps and 243 MB written per step.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
                     [--workload rollout65k|rollout1m|pixels16k|step4096|small64|
-                                cartpole65k|cartpole1m]
+                                cartpole65k|cartpole1m|policy65k]
 
 Prints one JSON line (rank 0).  With --gpus N > 1 it must be launched with
 torchrun, one rank per GPU; each rank simulates its own 65,536 envs (global env
@@ -68,6 +68,11 @@ WORKLOADS = {
         name="CartPole fused rollout, N=1048576 envs, T=32 steps per launch, in-kernel Philox actions",
         env="cartpole", n=1048576, T=32, mode=0, obs_mode=0, frameskip=1, bytes=21.0 + 48.0 / 32,
         kernel="k_cartpole_rollout", traffic=695.4e6),
+    "policy65k": dict(
+        name="policy in the loop: GRU policy (2.0 M parameters, bf16, cuBLAS) -> pong_sample_actions -> "
+             "pong_step, N=65536 envs, 32 agent steps per CUDA graph",
+        env="policy", n=65536, T=32, mode=2, obs_mode=0, frameskip=1, bytes=94.0 + 12.0 + 4.0 + 1.0,
+        kernel="cuBLAS GEMMs (library) + k_sample_actions + k_rollout_vector", traffic=None),
     "small64": dict(
         name="fused vector-obs rollout, N=64 envs, T=2000 steps per launch, in-kernel Philox actions",
         n=64, T=2000, mode=0, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 2000,
@@ -221,6 +226,106 @@ def run_reference(args, rank):
     }), flush=True)
 
 
+def run_policy(args, w, rank, world, local):
+    """The policy-in-the-loop workload: K agent steps per CUDA graph replay; a
+    "step" of the benchmark is one replay.  Also times the same graph without the
+    env-side kernels to report the env's share of the step."""
+    import torch
+    from paper_2603_12145_b200 import policy_loop, pong, sharding
+    import oracle
+    import numpy as np
+
+    N, K = w["n"], w["T"]
+    hidden = 576
+    steps = args.steps if args.steps > 0 else 100
+    warmup = max(args.warmup, 3)
+    env_id_base, _ = sharding.shard(rank, world, N)
+    policy = policy_loop.make_policy(hidden=hidden, seed=SEED, dtype=torch.bfloat16)
+    n_params = sum(p.numel() for p in policy.parameters())
+
+    def timed(with_env, with_policy=True):
+        loop = policy_loop.PolicyLoop(pong.PongEnv(N, SEED, env_id_base=env_id_base), policy, K)
+        loop.capture(with_env=with_env, with_policy=with_policy)
+        for _ in range(warmup):
+            loop.replay()
+        torch.cuda.synchronize()
+        l0 = loop.env.launches
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0 = time.perf_counter()
+        e0.record()
+        for _ in range(steps):
+            loop.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1), w0, time.perf_counter(), loop, loop.env.launches - l0
+
+    sampler = ClockSampler(physical_gpu_index(local))
+    sampler.start()
+    ms_env, w0, w1, loop, fill_launches = timed(True)
+    ms_pol, _, _, _, _ = timed(False)
+    ms_envk, _, _, _, _ = timed(True, with_policy=False)
+    # end to end: the step's metric (summed reward) is read back to the host after every replay
+    e2e_steps = max(args.e2e_steps, 1)
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        loop.replay()
+        float(loop.reward_sum.item())
+    e2e_s = time.perf_counter() - t0
+    sampler.stop()
+    ms_env = sharding.max_over_ranks(ms_env, device="cuda")
+    value = world * steps * N * K / (ms_env * 1e-3)
+    flops = 2.0 * n_params * N * K * steps
+    try:
+        peak_tf = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
+        peak_kind = "measured"
+    except Exception:
+        peak_tf, peak_kind = 1590.0, "fallback"
+    achieved_tf = flops / (ms_env * 1e-3) / 1e12
+    if rank != 0:
+        return
+    # CPU: the env-side part only (sampling from given logits + env step); the policy
+    # network has no oracle, it is a library call
+    n_s = 8192
+    o = oracle.OraclePong(n_s, SEED)
+    rng = np.random.Generator(np.random.PCG64(SEED))
+    logits = rng.normal(0, 1, (n_s, 3)).astype(np.float32)
+    c0, reps = time.perf_counter(), 0
+    while time.perf_counter() - c0 < max(args.cpu_seconds, 0.2):
+        words = o.fill_words(K)
+        for i in range(K):
+            o.step(oracle.sample_actions(logits, words[i]))
+        reps += 1
+    cpu_dt = time.perf_counter() - c0
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": ms_env / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16 policy, int32 env", "data": "synthetic",
+        "config": {"workload": w["name"], "workload_key": args.workload, "n_envs_per_gpu": N,
+                   "agent_steps_per_graph": K, "policy_parameters": n_params, "hidden": hidden,
+                   "env_steps_per_step": N * K,
+                   "l2": "the policy's activations and weights are read every step; no flush"},
+        "roofline": {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                     "frac": achieved_tf / peak_tf, "peak_source": peak_kind + " cuBLAS bf16",
+                     "traffic": None, "kernel": w["kernel"],
+                     "note": "the matrix products are cuBLAS library calls made by torch; 2 x parameters "
+                             "x envs flops per agent step"},
+        "policy_only_ms_per_step": ms_pol / steps,
+        "env_kernels_only_ms_per_step": ms_envk / steps,
+        "env_kernels_share_of_step": ms_envk / ms_env,
+        "env_and_bookkeeping_share_of_step": (ms_env - ms_pol) / ms_env,
+        "e2e": {"value": world * e2e_steps * N * K / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 8, "steps": e2e_steps,
+                "api": "PolicyLoop.replay + read-back of the summed reward"},
+        "gpu_launches": int(fill_launches + steps * K * 2),
+        "clocks": sampler.summary(w0, w1),
+        "cpu_baseline": {"value": reps * n_s * K / cpu_dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "host_cores": os.cpu_count(),
+                         "sample": "env-side part only (sampling from fixed logits + env step), envs "
+                                   "0..8191, %d x %d steps, %.1f s, single thread" % (reps, K, cpu_dt)},
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -256,6 +361,9 @@ def main():
     pong.load()
 
     w = WORKLOADS[args.workload]
+    if w.get("env") == "policy":
+        run_policy(args, w, rank, world, local)
+        return
     N, T, mode = w["n"], w["T"], w["mode"]
     pixels = w["obs_mode"] == 1
     env_steps_per_launch = N * T

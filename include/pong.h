@@ -159,6 +159,38 @@ int pong_rollout_host(pong_env *h, int T, int action_mode, const uint8_t *action
  * the global step. */
 int pong_fill_actions(pong_env *h, int T, int sticky, uint8_t *actions_out);
 
+/* ---- policy in the loop (the paper's "GRU rollout" setting: a policy network on
+ * the same stream produces the actions) ------------------------------------------
+ *
+ * pong_fill_words writes the Philox action words of global steps t .. t+T-1 to
+ * words_out (device uint32[T][n]); they are the uniform numbers of the draws
+ * below.  Does not advance the global step.
+ *
+ * pong_sample_actions draws one action per env from softmax(logits[i][0..2])
+ * (device float32[n][3], finite values) with the uniform number words[i] (device
+ * uint32[n]) and writes action bytes for pong_step to actions_out (device
+ * uint8[n]).  Everything is binary32 in a fixed order so that the draw is
+ * reproducible bit for bit:
+ *   m = max(l0,l1,l2); ei = expn(li - m); s = (e0 + e1) + e2;
+ *   x = ((float)(word >> 8) * 2^-24) * s;  a = x < e0 ? 0 : (x < e0 + e1 ? 1 : 2)
+ *   expn(x) = 2^f * 2^n with y = x * log2(e), n = floor(y + 0.5), f = y - n and
+ *   2^f = ((((((P6 f + P5) f + P4) f + P3) f + P2) f + P1) f + 1, Pk = ln(2)^k / k!
+ *   (0 when y < -150 or n < -126).
+ * It uses no state of the handle but its size and stream, so a captured launch
+ * can be replayed.
+ *
+ * pong_get_step_counter / pong_set_step_counter read and set the global agent
+ * step t.  They exist for captured launches: a CUDA graph replay runs the kernels
+ * but not the host code that counts steps, and capturing runs the host code but
+ * not the kernels, so the caller puts the counter right around both.  Only
+ * pong_step with vector observations is meant to be replayed that way: its
+ * kernel does not use the step number. */
+int pong_fill_words(pong_env *h, int T, uint32_t *words_out);
+int pong_sample_actions(pong_env *h, const float *logits, const uint32_t *words,
+                        uint8_t *actions_out);
+int pong_get_step_counter(pong_env *h, uint64_t *t);
+int pong_set_step_counter(pong_env *h, uint64_t t);
+
 /* Episodes finished since create / reset / the last clear: their number, the
  * sum of their returns (agent points - opponent points) and of their lengths
  * in frames.  Exact integers.  Outputs are HOST pointers (any may be NULL).

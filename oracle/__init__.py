@@ -262,9 +262,6 @@ class OraclePong:
         lib().oracle_fill_words(self.n, self.seed, self.env_id_base, self.t, int(T), _ptr(out))
         return out
 
-    def advance_step_counter(self, steps):
-        self.t += int(steps)
-
     def episode_stats(self, clear=False):
         s = (int(self.stats.episodes), int(self.stats.sum_return),
              int(self.stats.sum_length))

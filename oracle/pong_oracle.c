@@ -416,6 +416,7 @@ float oracle_expn(float x)
 {
     if (!(x <= 0.0f)) x = 0.0f;                 /* callers pass l - max <= 0; NaN -> 0 */
     float y = x * 1.44269504088896340736f;
+    if (y < -150.0f) return 0.0f;               /* far below 2^-126; keeps the int conversion in range */
     float t = y + 0.5f;
     float n = (float)(int)t;                    /* truncation towards zero ... */
     if (n > t) n = n - 1.0f;                    /* ... made a floor: n = round(y) */

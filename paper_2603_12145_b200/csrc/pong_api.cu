@@ -270,6 +270,41 @@ int pong_fill_actions(pong_env *h, int T, int sticky, uint8_t *actions_out)
     return PONG_OK;
 }
 
+int pong_fill_words(pong_env *h, int T, uint32_t *words_out)
+{
+    if (h == nullptr || words_out == nullptr) return PONG_ENULL;
+    if (T < 1 || (uint64_t)T * (uint64_t)h->n > (1ull << 40)) return PONG_EINVAL;
+    pong::LaunchArgs a = base_args(h);
+    a.T = T;
+    if (pong::launch_fill_words(a, words_out, h->stream) != cudaSuccess) return PONG_ECUDA;
+    const uint64_t groups = ((h->t + (uint64_t)T - 1) >> 2) - (h->t >> 2) + 1;
+    h->launches += (int64_t)((groups + 32767) / 32768);
+    return PONG_OK;
+}
+
+int pong_sample_actions(pong_env *h, const float *logits, const uint32_t *words, uint8_t *actions_out)
+{
+    if (h == nullptr || logits == nullptr || words == nullptr || actions_out == nullptr) return PONG_ENULL;
+    if (pong::launch_sample_actions(h->n, logits, words, actions_out, h->stream) != cudaSuccess)
+        return PONG_ECUDA;
+    h->launches += 1;
+    return PONG_OK;
+}
+
+int pong_get_step_counter(pong_env *h, uint64_t *t)
+{
+    if (h == nullptr || t == nullptr) return PONG_ENULL;
+    *t = h->t;
+    return PONG_OK;
+}
+
+int pong_set_step_counter(pong_env *h, uint64_t t)
+{
+    if (h == nullptr) return PONG_ENULL;
+    h->t = t;
+    return PONG_OK;
+}
+
 int pong_episode_stats(pong_env *h, int64_t *episodes, int64_t *sum_return, int64_t *sum_length,
                        int clear)
 {

@@ -707,4 +707,62 @@ cudaError_t launch_fill_actions(const LaunchArgs &a, int sticky, uint8_t *out, c
     return cudaSuccess;
 }
 
+// ---- policy interface ---------------------------------------------------------------------
+
+// Thread (x = env, y = Philox block): the four action words of steps 4g .. 4g+3.
+__global__ void __launch_bounds__(128) k_fill_words(const __grid_constant__ LaunchArgs a,
+                                                    uint32_t *__restrict__ out)
+{
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= a.n) return;
+    const unsigned long long t_begin = a.t0, t_end = a.t0 + (unsigned long long)a.T;
+    const unsigned long long g = (t_begin >> 2) + blockIdx.y;
+    uint32_t w[4];
+    action_words(g, a.env_id_base + (uint32_t)n, a.rk, w);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const unsigned long long tt = g * 4 + j;
+        if (tt >= t_begin && tt < t_end) out[(size_t)(tt - t_begin) * (size_t)a.n + (size_t)n] = w[j];
+    }
+}
+
+cudaError_t launch_fill_words(const LaunchArgs &a, uint32_t *out, cudaStream_t s)
+{
+    const unsigned long long g0 = a.t0 >> 2, g1 = (a.t0 + (unsigned long long)a.T - 1) >> 2;
+    const unsigned long long groups = g1 - g0 + 1;
+    LaunchArgs b = a;
+    unsigned long long done_groups = 0;
+    while (done_groups < groups) {  // gridDim.y is limited to 65535: slabs of whole Philox blocks
+        const unsigned long long slab = groups - done_groups < 32768ull ? groups - done_groups : 32768ull;
+        const unsigned long long slab_t0 = done_groups == 0 ? a.t0 : (g0 + done_groups) * 4;
+        unsigned long long slab_t1 = (g0 + done_groups + slab) * 4;
+        if (slab_t1 > a.t0 + (unsigned long long)a.T) slab_t1 = a.t0 + (unsigned long long)a.T;
+        b.t0 = slab_t0;
+        b.T = (int)(slab_t1 - slab_t0);
+        dim3 grid((a.n + 127) / 128, (unsigned)slab);
+        k_fill_words<<<grid, 128, 0, s>>>(b, out + (size_t)(slab_t0 - a.t0) * (size_t)a.n);
+        const cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+        done_groups += slab;
+    }
+    return cudaSuccess;
+}
+
+__global__ void __launch_bounds__(128) k_sample_actions(const int n, const float *__restrict__ logits,
+                                                        const uint32_t *__restrict__ words,
+                                                        uint8_t *__restrict__ out)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const float *l = logits + (size_t)i * 3;
+    out[i] = (uint8_t)sample_action(l[0], l[1], l[2], words[i]);
+}
+
+cudaError_t launch_sample_actions(int n, const float *logits, const uint32_t *words, uint8_t *out,
+                                  cudaStream_t s)
+{
+    k_sample_actions<<<(n + 127) / 128, 128, 0, s>>>(n, logits, words, out);
+    return cudaGetLastError();
+}
+
 }  // namespace pong

@@ -32,5 +32,8 @@ cudaError_t launch_reset(const LaunchArgs &a, cudaStream_t s);          // state
 cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s);
 cudaError_t launch_rollout_pixels(const LaunchArgs &a, int sm_count, cudaStream_t s);
 cudaError_t launch_fill_actions(const LaunchArgs &a, int sticky, uint8_t *out, cudaStream_t s);
+cudaError_t launch_fill_words(const LaunchArgs &a, uint32_t *out, cudaStream_t s);
+cudaError_t launch_sample_actions(int n, const float *logits, const uint32_t *words, uint8_t *out,
+                                  cudaStream_t s);
 
 }  // namespace pong

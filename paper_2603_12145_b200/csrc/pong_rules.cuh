@@ -349,6 +349,40 @@ __device__ __forceinline__ void philox_rounds(PhiloxPipe &p, const RoundKeys &rk
     }
 }
 
+// ---- policy interface: one action from three logits and one uniform word -------------
+// e^x for x <= 0 in binary32, fixed order: y = x*log2(e), n = round(y), f = y - n in
+// [-0.5, 0.5], 2^f by a degree-6 polynomial, scaled by 2^n through the exponent bits.
+__device__ __forceinline__ float expn(float x)
+{
+    if (!(x <= 0.0f)) x = 0.0f;
+    const float y = __fmul_rn(x, 1.44269504088896340736f);
+    if (y < -150.0f) return 0.0f;
+    const float n = floorf(__fadd_rn(y, 0.5f));
+    if (n < -126.0f) return 0.0f;
+    const float f = __fsub_rn(y, n);
+    float p = 1.5403530393381608e-4f;
+    p = __fadd_rn(__fmul_rn(p, f), 1.3333558146428443e-3f);
+    p = __fadd_rn(__fmul_rn(p, f), 9.6181291076284772e-3f);
+    p = __fadd_rn(__fmul_rn(p, f), 5.5504108664821580e-2f);
+    p = __fadd_rn(__fmul_rn(p, f), 2.4022650695910072e-1f);
+    p = __fadd_rn(__fmul_rn(p, f), 6.9314718055994531e-1f);
+    p = __fadd_rn(__fmul_rn(p, f), 1.0f);
+    return __fmul_rn(p, __int_as_float((__float2int_rn(n) + 127) << 23));
+}
+
+__device__ __forceinline__ int sample_action(float l0, float l1, float l2, uint32_t word)
+{
+    const float m = fmaxf(fmaxf(l0, l1), l2);
+    const float e0 = expn(__fsub_rn(l0, m));
+    const float e1 = expn(__fsub_rn(l1, m));
+    const float e2 = expn(__fsub_rn(l2, m));
+    const float e01 = __fadd_rn(e0, e1);
+    const float s = __fadd_rn(e01, e2);
+    const float u = __fmul_rn(__uint2float_rn(word >> 8), 5.9604644775390625e-08f);
+    const float x = __fmul_rn(u, s);
+    return x < e0 ? 0 : (x < e01 ? 1 : 2);
+}
+
 // ---- observations -----------------------------------------------------------------
 // float32(v) is exact (|v| < 2^24); one round-to-nearest multiply by
 // float32(1/40960) = 0x37CCCCCD.  Never a division, never fused.

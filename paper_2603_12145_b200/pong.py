@@ -24,7 +24,8 @@ FRAME_BYTES = 84 * 84
 EXPORTS = ("pong_create", "pong_create_ex", "pong_destroy", "pong_set_stream", "pong_reset",
            "pong_step", "pong_rollout", "pong_rollout_host", "pong_fill_actions",
            "pong_episode_stats", "pong_get_state", "pong_set_state", "pong_num_envs",
-           "pong_launch_count", "pong_strerror", "pong_rollout_static")
+           "pong_launch_count", "pong_strerror", "pong_rollout_static", "pong_fill_words",
+           "pong_sample_actions", "pong_get_step_counter", "pong_set_step_counter")
 STATIC_MAX_ENVS = 65536
 
 
@@ -69,6 +70,10 @@ def load(build_if_missing: bool = False):
     L.pong_rollout.argtypes = [vp, i32, i32, vp, vp, vp, vp]
     L.pong_rollout_host.argtypes = [vp, i32, i32, vp, vp, vp, vp]
     L.pong_fill_actions.argtypes = [vp, i32, i32, vp]
+    L.pong_fill_words.argtypes = [vp, i32, vp]
+    L.pong_sample_actions.argtypes = [vp, vp, vp, vp]
+    L.pong_get_step_counter.argtypes = [vp, ctypes.POINTER(u64)]
+    L.pong_set_step_counter.argtypes = [vp, u64]
     L.pong_episode_stats.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64),
                                      ctypes.POINTER(i64), i32]
     L.pong_get_state.argtypes = [vp, vp, ctypes.POINTER(u64)]
@@ -161,6 +166,25 @@ def pong_rollout_host(h: int, T: int, action_mode: int, actions_host, obs_host, 
 
 def pong_fill_actions(h: int, T: int, sticky: int, actions_out) -> None:
     _check(load().pong_fill_actions(h, int(T), int(sticky), _ptr(actions_out)), "pong_fill_actions")
+
+
+def pong_fill_words(h: int, T: int, words_out) -> None:
+    _check(load().pong_fill_words(h, int(T), _ptr(words_out)), "pong_fill_words")
+
+
+def pong_sample_actions(h: int, logits, words, actions_out) -> None:
+    _check(load().pong_sample_actions(h, _ptr(logits), _ptr(words), _ptr(actions_out)),
+           "pong_sample_actions")
+
+
+def pong_get_step_counter(h: int) -> int:
+    t = ctypes.c_uint64()
+    _check(load().pong_get_step_counter(h, ctypes.byref(t)), "pong_get_step_counter")
+    return int(t.value)
+
+
+def pong_set_step_counter(h: int, t: int) -> None:
+    _check(load().pong_set_step_counter(h, int(t)), "pong_set_step_counter")
 
 
 def pong_episode_stats(h: int, clear: bool = False) -> Tuple[int, int, int]:
@@ -289,6 +313,28 @@ class PongEnv:
             out = self.torch.empty((int(T), self.n), dtype=self.torch.uint8, device=self.device)
         pong_fill_actions(self.h, T, sticky, out)
         return out
+
+    def fill_words(self, T, out=None):
+        self._stream()
+        if out is None:
+            out = self.torch.empty((int(T), self.n), dtype=self.torch.int32, device=self.device)
+        pong_fill_words(self.h, T, out)
+        return out
+
+    def sample_actions(self, logits, words, out=None):
+        self._stream()
+        if out is None:
+            out = self.torch.empty((self.n,), dtype=self.torch.uint8, device=self.device)
+        pong_sample_actions(self.h, logits, words, out)
+        return out
+
+    @property
+    def t(self):
+        return pong_get_step_counter(self.h)
+
+    @t.setter
+    def t(self, value):
+        pong_set_step_counter(self.h, value)
 
     def episode_stats(self, clear=False):
         self._stream()
