@@ -350,6 +350,7 @@ static bool try_launch_vector_tma(const LaunchArgs &a, cudaStream_t s, cudaError
 {
     if (a.frameskip != 1) return false;
     if (a.n % 16 != 0 || a.t0 % 4 != 0 || a.T % kTmaStage != 0) return false;
+    if (a.n > (1 << 29)) return false;  // box origins 3 * n0 are 32-bit tensor coordinates
     const uintptr_t bases = reinterpret_cast<uintptr_t>(a.obs) | reinterpret_cast<uintptr_t>(a.reward) |
                             reinterpret_cast<uintptr_t>(a.done);
     if (bases % 16 != 0) return false;  // tensor maps need 16-byte aligned bases
