@@ -58,6 +58,26 @@ def test_rollout_every_mode_and_ragged_sizes(torch, n, mode):
     assert ora.episode_stats()[0] > 0
 
 
+@pytest.mark.parametrize("n", [16, 48, 64, 1040, 4096])
+@pytest.mark.parametrize("mode", [0, 2, 3])
+def test_aligned_sizes_and_long_rollouts(torch, n, mode):
+    """Batch sizes that are multiples of 16 with step counts that are and are not
+    multiples of 4, long enough for several refills of the start-state table."""
+    seed = 900 + n
+    env, ora = cp.CartPoleEnv(n, seed), ocp.OracleCartPole(n, seed)
+    for k, T in enumerate((8, 64, 16, 128, 200, 3, 8, 1, 24, 40, 512)):
+        if mode == 2:
+            a = actions(T, n, 50 + k)
+            g, o = env.rollout(T, 2, torch.from_numpy(a).cuda()), ora.rollout(T, 2, a)
+        elif mode == 3:
+            g, o = env.rollout(T, 3, k % 2), ora.rollout(T, 3, k % 2)
+        else:
+            g, o = env.rollout(T, 0), ora.rollout(T, 0)
+        assert_equal(g, o, "n %d mode %d T %d" % (n, mode, T))
+    assert_state_equal(env, ora)
+    assert ora.episode_stats()[0] > n
+
+
 def test_step_api_and_composition(torch):
     n, seed, T = 257, 6, 200
     env, ora = cp.CartPoleEnv(n, seed), ocp.OracleCartPole(n, seed)
