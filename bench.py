@@ -358,7 +358,7 @@ def main():
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    pong.load()
+    pong.load(build_if_missing=True)
 
     w = WORKLOADS[args.workload]
     if w.get("env") == "policy":
@@ -379,7 +379,7 @@ def main():
     obs_width = 4 if is_cartpole else 6
     if is_cartpole:
         from paper_2603_12145_b200 import cartpole
-        cartpole.load()
+        cartpole.load(build_if_missing=True)
         env = cartpole.CartPoleEnv(N, SEED, env_id_base=env_id_base)
         rollout_host = cartpole.cartpole_rollout_host
     else:

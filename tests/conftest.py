@@ -24,3 +24,19 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def _cuda_libraries_built():
+    """With a CUDA device present, compile the libraries that are missing or
+    older than their sources once per session, so that every GPU test loads the
+    hand-written kernels (there is no other path to fall back to)."""
+    try:
+        import torch
+        have = torch.cuda.is_available()
+    except Exception:
+        have = False
+    if have:
+        from paper_2603_12145_b200 import build
+        build.build()
+    yield

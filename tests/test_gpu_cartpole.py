@@ -14,7 +14,7 @@ pytestmark = pytest.mark.gpu
 def torch():
     import torch as t
     assert t.cuda.is_available()
-    cp.load()
+    cp.load(build_if_missing=True)
     return t
 
 

@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 def torch():
     import torch as t
     assert t.cuda.is_available()
-    pong.load()
+    pong.load(build_if_missing=True)
     return t
 
 

@@ -31,7 +31,7 @@ def run_both(torch, n, seed, base, T, mode):
 def test_static_rollout_matches_handle_rollout_twice_in_a_row():
     import torch
     assert torch.cuda.is_available()
-    pong.load()
+    pong.load(build_if_missing=True)
     # long enough for episodes to finish, so the counters are non-zero
     first = run_both(torch, 4096, 7, 0, 4000, pong.ACT_PHILOX)
     assert first[0] > 0
@@ -44,7 +44,7 @@ def test_static_rollout_matches_handle_rollout_twice_in_a_row():
 
 def test_static_rollout_rejects_bad_sizes():
     import torch
-    pong.load()
+    pong.load(build_if_missing=True)
     buf = torch.empty((64,), dtype=torch.float32, device="cuda")
     d = torch.empty((64,), dtype=torch.uint8, device="cuda")
     for n, code in ((pong.STATIC_MAX_ENVS + 1, -7), (0, -1)):
