@@ -50,3 +50,34 @@ def random_states(n_envs: int, seed: int, near_end: bool = False) -> np.ndarray:
     s[9] = rng.integers(0, 1000, n)                        # episode
     s[10] = rng.integers(0, 3, n)                          # prev_action
     return s
+
+
+def policy_weights(hidden: int, seed: int, obs_dim: int = 6, n_actions: int = 3) -> dict:
+    """float32 parameters of the GRU policy, rows = output units, gate blocks in
+    the order r, z, n.  Every matrix entry is an integer / 2048 with at most
+    seven significant bits, so it is exactly representable in bfloat16 and both
+    the tensor-core path and the CPU oracle see the same numbers; the range
+    matches the usual 1 / sqrt(hidden) initialisation at hidden = 576."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    H = hidden
+
+    def m(*shape):
+        return (rng.integers(-85, 86, size=shape).astype(np.float32) / np.float32(2048.0))
+
+    return {
+        "enc_w": (rng.integers(-96, 97, size=(H, obs_dim)).astype(np.float32) / np.float32(64.0)),
+        "enc_b": m(H),
+        "w_ih": m(3 * H, H), "w_hh": m(3 * H, H), "b_ih": m(3 * H), "b_hh": m(3 * H),
+        "head_w": (rng.integers(-96, 97, size=(n_actions, H)).astype(np.float32)
+                   / np.float32(512.0)),
+        "head_b": m(n_actions),
+    }
+
+
+def policy_activations(n_envs: int, hidden: int, seed: int):
+    """(x, h): float32 [n_envs, hidden] each, bfloat16-representable values; x is
+    non-negative like an encoder output after its rectifier, h lies in (-1, 1)."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    x = rng.integers(0, 128, size=(n_envs, hidden)).astype(np.float32) / np.float32(64.0)
+    h = rng.integers(-127, 128, size=(n_envs, hidden)).astype(np.float32) / np.float32(128.0)
+    return x, h
