@@ -17,9 +17,11 @@ TARGETS = {
     "libpong_b200.so": (["pong_api.cu", "pong_kernels.cu", "pong_noalloc.cu"],
                         ["pong_rules.cuh", "pong_kernels.cuh", os.path.join(INCLUDE, "pong.h")]),
     "libcartpole_b200.so": (["cartpole.cu"], [os.path.join(INCLUDE, "cartpole.h")]),
+    "libgru_policy_b200.so": (["gru_policy.cu"], [os.path.join(INCLUDE, "gru_policy.h")]),
 }
 LIB = os.path.join(HERE, "libpong_b200.so")
 CARTPOLE_LIB = os.path.join(HERE, "libcartpole_b200.so")
+GRU_POLICY_LIB = os.path.join(HERE, "libgru_policy_b200.so")
 
 
 def _nvcc() -> str:
@@ -71,3 +73,4 @@ if __name__ == "__main__":
     build(force=True, verbose="-v" in sys.argv)
     print(LIB)
     print(CARTPOLE_LIB)
+    print(GRU_POLICY_LIB)

@@ -1,0 +1,760 @@
+// gru_policy.cu -- the recurrent policy of the policy-in-the-loop rollout (the
+// paper's "GRU rollout (~2M parameters)" setting, Table "PufferLib comparisons";
+// Sec. 4, time breakdown) as sm_100a kernels behind the C ABI of gru_policy.h.
+//
+// k_gru_cell is the dense part: per 128-env tile and 64-unit slice of the hidden
+// state it forms the four pre-activation blocks
+//     nx = x W_in^T        r = x W_ir^T + h W_hr^T
+//     nh = h W_hn^T        z = x W_iz^T + h W_hz^T
+// on the tensor cores (tcgen05.mma, bfloat16 operands staged in shared memory by
+// TMA with the 128-byte swizzle, binary32 accumulators in tensor memory) and
+// applies biases, gates and the blend in the epilogue straight out of tensor
+// memory.  The weights are packed at create time so that one 192-row box holds
+// the three gate blocks a stage needs: [n | r | z] rows for the x half of the
+// reduction, [r | z | n] for the h half.  With the accumulator columns laid out
+// as [nx | r | z | nh], the x half is one N = 192 instruction into columns 0..191
+// and the h half one N = 192 instruction into columns 64..255, so r and z collect
+// both halves and the two candidate parts stay separate, as the reset gate needs.
+//
+// Roles in a 192-thread block (one block per SM, persistent over tiles):
+//   warp 0    TMA producer (one lane): fills a 5-deep ring of {x|h tile, weight box}
+//   warp 1    allocates tensor memory; one lane issues the MMAs and commits
+//   warps 2-5 epilogue: tcgen05.ld, gates, bfloat16 store; two accumulator
+//             buffers (2 x 256 columns) let it overlap the next tile's MMAs
+// Every mbarrier wait is bounded by a wall-clock limit; a wait that runs out
+// raises the block's abort flag, all roles leave their loops, the error word is
+// set and the block still frees its tensor memory.
+#include <cstdint>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "../../include/gru_policy.h"
+
+namespace {
+
+constexpr int kBM = 128;                         // envs per tile (MMA M)
+constexpr int kBK = 64;                          // reduction elements per stage = one 128-byte row
+constexpr int kHT = 64;                          // hidden units per tile
+constexpr int kBN = 3 * kHT;                     // weight rows per stage (MMA N)
+constexpr int kStages = 5;
+constexpr int kABytes = kBM * kBK * 2;           // 16 KB
+constexpr int kBBytes = kBN * kBK * 2;           // 24 KB
+constexpr int kStageBytes = kABytes + kBBytes;   // 40 KB
+constexpr int kAccCols = 4 * kHT;                // one accumulator buffer: nx | r | z | nh
+constexpr int kTmemCols = 2 * kAccCols;          // 512: all of tensor memory
+constexpr int kCellThreads = 192;
+constexpr int kBarrierBytes = 256;
+constexpr int kCellSmem = kStages * kStageBytes + kBarrierBytes + 1024;  // + slack to align to 1024
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait
+constexpr unsigned long long kDrainNs = 200000ull;          // let copies in flight land after an abort
+
+static_assert(kTmemCols == 512, "two accumulator buffers fill tensor memory");
+static_assert(kStageBytes % 1024 == 0 && kABytes % 1024 == 0, "swizzled tiles need 1024-byte alignment");
+
+// ---------------------------------------------------------------- PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+
+// Waits for the phase of the given parity to complete.  Gives up (and raises the
+// block's abort flag) after kWaitLimitNs, or as soon as another role has raised it.
+__device__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 0;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 63u) {
+            if (*abort_flag) return false;
+            const unsigned long long now = global_timer_ns();
+            if (t0 == 0) {
+                t0 = now;
+            } else if (now - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before_sync()
+{
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+
+__device__ __forceinline__ void tc_fence_after_sync()
+{
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot),
+                 "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
+                 : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, bfloat16 operands, binary32 accumulate.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                          uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// The mbarrier receives one arrival once every MMA issued so far by this thread is done.
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+                 : "memory");
+}
+
+// 16 consecutive accumulator columns of this thread's lane.
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, "
+        "%12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_wait_ld()
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory operand descriptor of a K-major tile whose rows are 128 bytes
+// (64 bfloat16) with the 128-byte swizzle, as TMA writes it: 8-row groups are
+// 1024 bytes apart (stride offset), the leading offset is not used by swizzled
+// K-major layouts (set to 1), descriptor version 1, layout type 2 = 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
+{
+    return static_cast<uint64_t>((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+
+// Instruction descriptor: binary32 accumulator, bfloat16 A and B, both K-major, M = 128.
+__host__ __device__ constexpr uint32_t instr_desc(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+           (static_cast<uint32_t>(kBM >> 4) << 24);
+}
+
+__device__ __forceinline__ float sigmoid_f(float v)
+{
+    return __fdividef(1.0f, 1.0f + __expf(-v));
+}
+
+__device__ __forceinline__ float tanh_f(float v)
+{
+    return 1.0f - __fdividef(2.0f, __expf(2.0f * v) + 1.0f);
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+
+struct CellArgs {
+    const __nv_bfloat16 *h_in;
+    __nv_bfloat16 *h_out;
+    const float *b_r;   // b_ir + b_hr
+    const float *b_z;   // b_iz + b_hz
+    const float *b_in;
+    const float *b_hn;
+    int n;
+    int H;
+    int *err;
+};
+
+// ---------------------------------------------------------------- the cell
+
+__global__ void __launch_bounds__(kCellThreads, 1)
+k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_h,
+           const __grid_constant__ CUtensorMap tm_wx, const __grid_constant__ CUtensorMap tm_wh,
+           const CellArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t tiles = (raw + 1023u) & ~1023u;           // stage ring, 1024-byte aligned
+    const uint32_t bars = tiles + kStages * kStageBytes;     // mbarriers, 8 bytes each
+    uint8_t *bars_ptr = smem_raw + (bars - raw);
+    const uint32_t full0 = bars, empty0 = bars + 8 * kStages;
+    const uint32_t acc_full0 = bars + 16 * kStages, acc_empty0 = acc_full0 + 16;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars_ptr + 16 * kStages + 32);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_ptr + 16 * kStages + 40);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int KC = a.H / kBK;                 // reduction chunks per half
+    const int JT = a.H / kHT;                 // hidden tiles
+    const int m_tiles = (a.n + kBM - 1) / kBM;
+    const int n_tasks = m_tiles * JT;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(acc_full0 + 8 * b, 1);
+            mbar_init(acc_empty0 + 8 * b, 4);   // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x) {
+                const int mt = task / JT, j = task - mt * JT;
+                for (int half = 0; half < 2 && ok; ++half) {
+                    const CUtensorMap *ta = half ? &tm_h : &tm_x;
+                    const CUtensorMap *tb = half ? &tm_wh : &tm_wx;
+                    for (int kc = 0; kc < KC; ++kc) {
+                        if (!mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        const uint32_t dst = tiles + s * kStageBytes;
+                        mbar_expect_tx(full0 + 8 * s, kStageBytes);
+                        tma_load_2d(dst, ta, kc * kBK, mt * kBM, full0 + 8 * s);
+                        tma_load_2d(dst + kABytes, tb, kc * kBK, j * kBN, full0 + 8 * s);
+                        if (++s == kStages) {
+                            s = 0;
+                            ph ^= 1u;
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t kIdesc192 = instr_desc(kBN);
+            constexpr uint32_t kIdesc128 = instr_desc(2 * kHT);
+            constexpr uint32_t kIdesc64 = instr_desc(kHT);
+            uint32_t s = 0, ph = 0;
+            bool ok = true;
+            int it = 0;
+            for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x, ++it) {
+                const uint32_t buf = it & 1, use = (it >> 1) & 1;
+                if (!mbar_wait(acc_empty0 + 8 * buf, use ^ 1u, abort_flag)) break;
+                tc_fence_after_sync();
+                const uint32_t d = tmem_base + buf * kAccCols;
+                for (int half = 0; half < 2 && ok; ++half) {
+                    for (int kc = 0; kc < KC; ++kc) {
+                        if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after_sync();
+                        const uint32_t a_addr = tiles + s * kStageBytes;
+                        const uint64_t ad = smem_desc(a_addr), bd = smem_desc(a_addr + kABytes);
+#pragma unroll
+                        for (int k = 0; k < kBK / 16; ++k) {
+                            // 16 elements = 32 bytes further along the swizzled row: +2 in the address field
+                            const uint64_t ak = ad + 2u * k, bk = bd + 2u * k;
+                            if (half == 0) {
+                                umma_bf16(d, ak, bk, kIdesc192, (kc | k) != 0);
+                            } else if ((kc | k) == 0) {
+                                // first step of the h half: r and z already hold the x half, nh starts here
+                                umma_bf16(d + kHT, ak, bk, kIdesc128, 1u);
+                                umma_bf16(d + 3 * kHT, ak, bk + ((2 * kHT * 128) >> 4), kIdesc64, 0u);
+                            } else {
+                                umma_bf16(d + kHT, ak, bk, kIdesc192, 1u);
+                            }
+                        }
+                        umma_commit(empty0 + 8 * s);   // the stage is free once these MMAs have read it
+                        if (++s == kStages) {
+                            s = 0;
+                            ph ^= 1u;
+                        }
+                    }
+                }
+                if (ok) umma_commit(acc_full0 + 8 * buf);
+            }
+        }
+    } else {
+        const int q = warp & 3;                       // the quarter of the lanes this warp may read
+        const int row_in_tile = q * 32 + lane;
+        int it = 0;
+        for (int task = blockIdx.x; task < n_tasks; task += gridDim.x, ++it) {
+            const int mt = task / JT, j = task - mt * JT;
+            const uint32_t buf = it & 1, use = (it >> 1) & 1;
+            const bool ready = mbar_wait(acc_full0 + 8 * buf, use, abort_flag);
+            if (!__all_sync(0xFFFFFFFFu, ready)) break;
+            tc_fence_after_sync();
+            const long long row = static_cast<long long>(mt) * kBM + row_in_tile;
+            const bool live = row < a.n;
+            const uint32_t t0 = tmem_base + buf * kAccCols + (static_cast<uint32_t>(q * 32) << 16);
+            const size_t off = static_cast<size_t>(live ? row : 0) * a.H + static_cast<size_t>(j) * kHT;
+            const uint4 *hrow = reinterpret_cast<const uint4 *>(a.h_in + off);
+            uint4 *orow = reinterpret_cast<uint4 *>(a.h_out + off);
+            const int col0 = j * kHT;
+#pragma unroll 1
+            for (int c = 0; c < kHT; c += 16) {
+                uint32_t nx[16], r[16], z[16], nh[16];
+                tmem_ld16(t0 + c, nx);
+                tmem_ld16(t0 + kHT + c, r);
+                tmem_ld16(t0 + 2 * kHT + c, z);
+                tmem_ld16(t0 + 3 * kHT + c, nh);
+                uint4 hv[2];
+                hv[0] = live ? __ldg(hrow + c / 8) : make_uint4(0, 0, 0, 0);
+                hv[1] = live ? __ldg(hrow + c / 8 + 1) : make_uint4(0, 0, 0, 0);
+                tmem_wait_ld();
+                const uint32_t hw[8] = {hv[0].x, hv[0].y, hv[0].z, hv[0].w,
+                                        hv[1].x, hv[1].y, hv[1].z, hv[1].w};
+                uint32_t ow[8];
+#pragma unroll
+                for (int i = 0; i < 16; i += 2) {
+                    float o[2];
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int col = col0 + c + i + e;
+                        const float rr = sigmoid_f(__uint_as_float(r[i + e]) + __ldg(a.b_r + col));
+                        const float zz = sigmoid_f(__uint_as_float(z[i + e]) + __ldg(a.b_z + col));
+                        const float cand = tanh_f(__uint_as_float(nx[i + e]) + __ldg(a.b_in + col) +
+                                                  rr * (__uint_as_float(nh[i + e]) + __ldg(a.b_hn + col)));
+                        const float hold = e ? bf16_hi(hw[i / 2]) : bf16_lo(hw[i / 2]);
+                        o[e] = cand + zz * (hold - cand);
+                    }
+                    ow[i / 2] = pack_bf16(o[0], o[1]);
+                }
+                if (live) {
+                    orow[c / 8] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+                    orow[c / 8 + 1] = make_uint4(ow[4], ow[5], ow[6], ow[7]);
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty0 + 8 * buf);
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait ran out: report it, then give copies that may still be in flight time to land
+        if (threadIdx.x == 0) atomicExch(a.err, 1);
+        const unsigned long long t0 = global_timer_ns();
+        while (global_timer_ns() - t0 < kDrainNs) __nanosleep(1000);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---------------------------------------------------------------- encoder and head
+
+// One thread per (env, 8 hidden units): x = bf16(relu(fma chain)), one 16-byte store;
+// also clears the same 8 units of h where the env's episode just ended.
+__global__ void __launch_bounds__(256)
+k_encode(const float *__restrict__ obs, const uint8_t *__restrict__ done, __nv_bfloat16 *__restrict__ h,
+         __nv_bfloat16 *__restrict__ x_out, const float *__restrict__ enc_w,
+         const float *__restrict__ enc_b, int n, int H, int obs_dim)
+{
+    const int groups = H / 8;
+    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (idx >= static_cast<long long>(n) * groups) return;
+    const int m = static_cast<int>(idx / groups), g = static_cast<int>(idx - static_cast<long long>(m) * groups);
+    float o[GRU_POLICY_MAX_OBS];
+#pragma unroll
+    for (int i = 0; i < GRU_POLICY_MAX_OBS; ++i)
+        o[i] = i < obs_dim ? __ldg(obs + static_cast<size_t>(m) * obs_dim + i) : 0.0f;
+    uint32_t w[4];
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+        float v[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int c = g * 8 + 2 * p + e;
+            float acc = __ldg(enc_b + c);
+#pragma unroll
+            for (int i = 0; i < GRU_POLICY_MAX_OBS; ++i)
+                if (i < obs_dim) acc = __fmaf_rn(o[i], __ldg(enc_w + static_cast<size_t>(c) * obs_dim + i), acc);
+            v[e] = acc > 0.0f ? acc : 0.0f;
+        }
+        w[p] = pack_bf16(v[0], v[1]);
+    }
+    const size_t off = static_cast<size_t>(m) * H + static_cast<size_t>(g) * 8;
+    *reinterpret_cast<uint4 *>(x_out + off) = make_uint4(w[0], w[1], w[2], w[3]);
+    if (done != nullptr && h != nullptr && __ldg(done + m) != 0)
+        *reinterpret_cast<uint4 *>(h + off) = make_uint4(0, 0, 0, 0);
+}
+
+// One thread per env: logits[a] = fma chain over the hidden units in ascending order.
+__global__ void __launch_bounds__(128)
+k_head(const __nv_bfloat16 *__restrict__ h, float *__restrict__ logits, const float *__restrict__ head_w,
+       const float *__restrict__ head_b, int n, int H, int A)
+{
+    extern __shared__ float w_s[];   // [A][H]
+    for (int i = threadIdx.x; i < A * H; i += blockDim.x) w_s[i] = head_w[i];
+    __syncthreads();
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= n) return;
+    float acc[GRU_POLICY_MAX_ACTIONS];
+#pragma unroll
+    for (int a = 0; a < GRU_POLICY_MAX_ACTIONS; ++a) acc[a] = a < A ? __ldg(head_b + a) : 0.0f;
+    const uint4 *row = reinterpret_cast<const uint4 *>(h + static_cast<size_t>(m) * H);
+    for (int k8 = 0; k8 < H / 8; ++k8) {
+        const uint4 v = __ldg(row + k8);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const float lo = bf16_lo(w[p]), hi = bf16_hi(w[p]);
+            const int k = k8 * 8 + 2 * p;
+#pragma unroll
+            for (int a = 0; a < GRU_POLICY_MAX_ACTIONS; ++a)
+                if (a < A) {
+                    acc[a] = __fmaf_rn(lo, w_s[a * H + k], acc[a]);
+                    acc[a] = __fmaf_rn(hi, w_s[a * H + k + 1], acc[a]);
+                }
+        }
+    }
+#pragma unroll
+    for (int a = 0; a < GRU_POLICY_MAX_ACTIONS; ++a)
+        if (a < A) logits[static_cast<size_t>(m) * A + a] = acc[a];
+}
+
+// ---------------------------------------------------------------- host side
+
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                      const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                      const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder, looked up once through the runtime (no link
+// against libcuda); nullptr if this driver does not have it.
+TensorMapEncodeFn tensor_map_encoder()
+{
+    static TensorMapEncodeFn fn = []() -> TensorMapEncodeFn {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        return reinterpret_cast<TensorMapEncodeFn>(p);
+    }();
+    return fn;
+}
+
+// bfloat16 [rows][H] row-major, boxes of 64 elements x box_rows rows, 128-byte swizzle;
+// rows past the end read as zero.
+bool encode_operand(TensorMapEncodeFn enc, CUtensorMap *m, const void *base, uint64_t H, uint64_t rows,
+                    uint32_t box_rows)
+{
+    const cuuint64_t dims[2] = {H, rows};
+    const cuuint64_t strides[1] = {H * 2};
+    const cuuint32_t box[2] = {kBK, box_rows};
+    const cuuint32_t elem_strides[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box,
+               elem_strides, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+struct gru_policy {
+    int H = 0, obs_dim = 0, A = 0;
+    int device = 0, sms = 0;
+    cudaStream_t stream = nullptr;
+    int64_t launches = 0;
+    __nv_bfloat16 *wx = nullptr, *wh = nullptr;   // packed [H/64][192][H]
+    float *b_r = nullptr, *b_z = nullptr, *b_in = nullptr, *b_hn = nullptr;
+    float *enc_w = nullptr, *enc_b = nullptr, *head_w = nullptr, *head_b = nullptr;
+    int *err = nullptr;
+    CUtensorMap tm_wx, tm_wh;
+};
+
+namespace {
+
+template <typename T>
+bool upload(T **dst, const std::vector<T> &src)
+{
+    if (cudaMalloc(reinterpret_cast<void **>(dst), src.size() * sizeof(T)) != cudaSuccess) return false;
+    return cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice) == cudaSuccess;
+}
+
+void release(gru_policy *p)
+{
+    cudaFree(p->wx);
+    cudaFree(p->wh);
+    cudaFree(p->b_r);
+    cudaFree(p->b_z);
+    cudaFree(p->b_in);
+    cudaFree(p->b_hn);
+    cudaFree(p->enc_w);
+    cudaFree(p->enc_b);
+    cudaFree(p->head_w);
+    cudaFree(p->head_b);
+    cudaFree(p->err);
+    delete p;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions, const float *enc_w,
+                      const float *enc_b, const float *w_ih, const float *w_hh, const float *b_ih,
+                      const float *b_hh, const float *head_w, const float *head_b)
+{
+    if (out == nullptr) return GRU_POLICY_ENULL;
+    *out = nullptr;
+    if (!enc_w || !enc_b || !w_ih || !w_hh || !b_ih || !b_hh || !head_w || !head_b) return GRU_POLICY_ENULL;
+    if (hidden < 64 || hidden > GRU_POLICY_MAX_HIDDEN || hidden % 64 != 0) return GRU_POLICY_EINVAL;
+    if (obs_dim < 1 || obs_dim > GRU_POLICY_MAX_OBS) return GRU_POLICY_EINVAL;
+    if (n_actions < 1 || n_actions > GRU_POLICY_MAX_ACTIONS) return GRU_POLICY_EINVAL;
+    if (tensor_map_encoder() == nullptr) return GRU_POLICY_ECUDA;
+    gru_policy *p = new (std::nothrow) gru_policy;
+    if (p == nullptr) return GRU_POLICY_ENOMEM;
+    const int H = hidden;
+    p->H = H;
+    p->obs_dim = obs_dim;
+    p->A = n_actions;
+    cudaDeviceProp prop;
+    if (cudaGetDevice(&p->device) != cudaSuccess ||
+        cudaGetDeviceProperties(&prop, p->device) != cudaSuccess) {
+        cudaGetLastError();
+        delete p;
+        return GRU_POLICY_ECUDA;
+    }
+    p->sms = prop.multiProcessorCount;
+
+    // Pack the weights: tile j holds, for the x half, rows [W_in | W_ir | W_iz] of its 64 units
+    // and, for the h half, rows [W_hr | W_hz | W_hn]; gate blocks of the inputs are r, z, n.
+    const int JT = H / kHT;
+    std::vector<__nv_bfloat16> wx(static_cast<size_t>(3) * H * H), wh(wx.size());
+    const int x_gate[3] = {2, 0, 1}, h_gate[3] = {0, 1, 2};
+    for (int j = 0; j < JT; ++j)
+        for (int g = 0; g < 3; ++g)
+            for (int i = 0; i < kHT; ++i) {
+                const size_t dst = (static_cast<size_t>(j) * kBN + g * kHT + i) * H;
+                const size_t sx = (static_cast<size_t>(x_gate[g]) * H + j * kHT + i) * H;
+                const size_t sh = (static_cast<size_t>(h_gate[g]) * H + j * kHT + i) * H;
+                for (int k = 0; k < H; ++k) {
+                    wx[dst + k] = __float2bfloat16_rn(w_ih[sx + k]);
+                    wh[dst + k] = __float2bfloat16_rn(w_hh[sh + k]);
+                }
+            }
+    std::vector<float> b_r(H), b_z(H), b_in(H), b_hn(H);
+    for (int c = 0; c < H; ++c) {
+        b_r[c] = b_ih[c] + b_hh[c];
+        b_z[c] = b_ih[H + c] + b_hh[H + c];
+        b_in[c] = b_ih[2 * H + c];
+        b_hn[c] = b_hh[2 * H + c];
+    }
+    bool ok = upload(&p->wx, wx) && upload(&p->wh, wh) && upload(&p->b_r, b_r) && upload(&p->b_z, b_z) &&
+              upload(&p->b_in, b_in) && upload(&p->b_hn, b_hn) &&
+              upload(&p->enc_w, std::vector<float>(enc_w, enc_w + static_cast<size_t>(H) * obs_dim)) &&
+              upload(&p->enc_b, std::vector<float>(enc_b, enc_b + H)) &&
+              upload(&p->head_w, std::vector<float>(head_w, head_w + static_cast<size_t>(n_actions) * H)) &&
+              upload(&p->head_b, std::vector<float>(head_b, head_b + n_actions)) &&
+              upload(&p->err, std::vector<int>(1, 0));
+    if (ok) {
+        TensorMapEncodeFn enc = tensor_map_encoder();
+        ok = encode_operand(enc, &p->tm_wx, p->wx, H, static_cast<uint64_t>(3) * H, kBN) &&
+             encode_operand(enc, &p->tm_wh, p->wh, H, static_cast<uint64_t>(3) * H, kBN);
+    }
+    if (ok) ok = cudaFuncSetAttribute(k_gru_cell, cudaFuncAttributeMaxDynamicSharedMemorySize, kCellSmem) ==
+                 cudaSuccess;
+    if (ok && static_cast<size_t>(n_actions) * H * sizeof(float) > 48 * 1024)
+        ok = cudaFuncSetAttribute(k_head, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  static_cast<int>(n_actions * H * sizeof(float))) == cudaSuccess;
+    if (!ok) {
+        cudaGetLastError();
+        release(p);
+        return GRU_POLICY_ECUDA;
+    }
+    *out = p;
+    return GRU_POLICY_OK;
+}
+
+int gru_policy_destroy(gru_policy *p)
+{
+    if (p == nullptr) return GRU_POLICY_ENULL;
+    cudaStreamSynchronize(p->stream);
+    release(p);
+    return GRU_POLICY_OK;
+}
+
+int gru_policy_set_stream(gru_policy *p, void *cuda_stream)
+{
+    if (p == nullptr) return GRU_POLICY_ENULL;
+    p->stream = static_cast<cudaStream_t>(cuda_stream);
+    return GRU_POLICY_OK;
+}
+
+int gru_policy_encode(gru_policy *p, const float *obs, const uint8_t *done, void *h, void *x_out, int n)
+{
+    if (p == nullptr || obs == nullptr || x_out == nullptr) return GRU_POLICY_ENULL;
+    if (n < 1) return GRU_POLICY_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(x_out) | reinterpret_cast<uintptr_t>(h)) % 16 != 0) return GRU_POLICY_EALIGN;
+    const long long threads = static_cast<long long>(n) * (p->H / 8);
+    const unsigned blocks = static_cast<unsigned>((threads + 255) / 256);
+    k_encode<<<blocks, 256, 0, p->stream>>>(obs, done, static_cast<__nv_bfloat16 *>(h),
+                                             static_cast<__nv_bfloat16 *>(x_out), p->enc_w, p->enc_b, n,
+                                             p->H, p->obs_dim);
+    if (cudaGetLastError() != cudaSuccess) return GRU_POLICY_ECUDA;
+    p->launches += 1;
+    return GRU_POLICY_OK;
+}
+
+int gru_policy_cell(gru_policy *p, const void *x, const void *h_in, void *h_out, int n)
+{
+    if (p == nullptr || x == nullptr || h_in == nullptr || h_out == nullptr) return GRU_POLICY_ENULL;
+    if (n < 1) return GRU_POLICY_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(h_in) |
+         reinterpret_cast<uintptr_t>(h_out)) % 16 != 0)
+        return GRU_POLICY_EALIGN;
+    if (h_out == x || h_out == h_in) return GRU_POLICY_EINVAL;
+    TensorMapEncodeFn enc = tensor_map_encoder();
+    CUtensorMap tm_x, tm_h;
+    if (!encode_operand(enc, &tm_x, x, p->H, n, kBM) || !encode_operand(enc, &tm_h, h_in, p->H, n, kBM))
+        return GRU_POLICY_ECUDA;
+    CellArgs a;
+    a.h_in = static_cast<const __nv_bfloat16 *>(h_in);
+    a.h_out = static_cast<__nv_bfloat16 *>(h_out);
+    a.b_r = p->b_r;
+    a.b_z = p->b_z;
+    a.b_in = p->b_in;
+    a.b_hn = p->b_hn;
+    a.n = n;
+    a.H = p->H;
+    a.err = p->err;
+    const long long tasks = static_cast<long long>((n + kBM - 1) / kBM) * (p->H / kHT);
+    const unsigned blocks = static_cast<unsigned>(tasks < p->sms ? tasks : p->sms);
+    k_gru_cell<<<blocks, kCellThreads, kCellSmem, p->stream>>>(tm_x, tm_h, p->tm_wx, p->tm_wh, a);
+    if (cudaGetLastError() != cudaSuccess) return GRU_POLICY_ECUDA;
+    p->launches += 1;
+    return GRU_POLICY_OK;
+}
+
+int gru_policy_head(gru_policy *p, const void *h, float *logits, int n)
+{
+    if (p == nullptr || h == nullptr || logits == nullptr) return GRU_POLICY_ENULL;
+    if (n < 1) return GRU_POLICY_EINVAL;
+    if (reinterpret_cast<uintptr_t>(h) % 16 != 0) return GRU_POLICY_EALIGN;
+    const unsigned blocks = static_cast<unsigned>((n + 127) / 128);
+    k_head<<<blocks, 128, static_cast<size_t>(p->A) * p->H * sizeof(float), p->stream>>>(
+        static_cast<const __nv_bfloat16 *>(h), logits, p->head_w, p->head_b, n, p->H, p->A);
+    if (cudaGetLastError() != cudaSuccess) return GRU_POLICY_ECUDA;
+    p->launches += 1;
+    return GRU_POLICY_OK;
+}
+
+int gru_policy_status(gru_policy *p)
+{
+    if (p == nullptr) return GRU_POLICY_ENULL;
+    if (cudaStreamSynchronize(p->stream) != cudaSuccess) return GRU_POLICY_ECUDA;
+    int flag = 0;
+    if (cudaMemcpy(&flag, p->err, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return GRU_POLICY_ECUDA;
+    if (flag != 0) {
+        cudaMemset(p->err, 0, sizeof(int));
+        return GRU_POLICY_ETIMEOUT;
+    }
+    return GRU_POLICY_OK;
+}
+
+int gru_policy_hidden(const gru_policy *p) { return p ? p->H : GRU_POLICY_ENULL; }
+
+int64_t gru_policy_launch_count(const gru_policy *p) { return p ? p->launches : 0; }
+
+const char *gru_policy_strerror(int code)
+{
+    switch (code) {
+    case GRU_POLICY_OK: return "ok";
+    case GRU_POLICY_EINVAL: return "invalid size or overlapping buffers";
+    case GRU_POLICY_ENULL: return "required pointer is NULL";
+    case GRU_POLICY_EALIGN: return "x / h pointer not 16-byte aligned";
+    case GRU_POLICY_ECUDA: return "CUDA runtime call or launch failed";
+    case GRU_POLICY_ENOMEM: return "allocation failed";
+    case GRU_POLICY_ETIMEOUT: return "a kernel gave up a bounded wait; its output is invalid";
+    default: return "unknown error";
+    }
+}
+
+}  // extern "C"

@@ -81,3 +81,14 @@ def policy_activations(n_envs: int, hidden: int, seed: int):
     x = rng.integers(0, 128, size=(n_envs, hidden)).astype(np.float32) / np.float32(64.0)
     h = rng.integers(-127, 128, size=(n_envs, hidden)).astype(np.float32) / np.float32(128.0)
     return x, h
+
+
+def bf16_values(shape, seed: int, min_exp: int = -6, max_exp: int = 0) -> np.ndarray:
+    """float32 array of random bfloat16-representable values +-(1 + m/128) * 2^e,
+    m uniform on 0..127 and e uniform on min_exp..max_exp, assembled from the bit
+    fields (no rounding involved)."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    sign = rng.integers(0, 2, size=shape, dtype=np.uint32) << np.uint32(31)
+    expo = (rng.integers(min_exp, max_exp + 1, size=shape) + 127).astype(np.uint32) << np.uint32(23)
+    mant = rng.integers(0, 128, size=shape, dtype=np.uint32) << np.uint32(16)
+    return (sign | expo | mant).view(np.float32)
