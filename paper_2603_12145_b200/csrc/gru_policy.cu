@@ -16,11 +16,13 @@
 // and the h half one N = 192 instruction into columns 64..255, so r and z collect
 // both halves and the two candidate parts stay separate, as the reset gate needs.
 //
-// Roles in a 192-thread block (one block per SM, persistent over tiles):
+// Roles in a 320-thread block (one block per SM, persistent over tiles):
 //   warp 0    TMA producer (one lane): fills a 5-deep ring of {x|h tile, weight box}
 //   warp 1    allocates tensor memory; one lane issues the MMAs and commits
-//   warps 2-5 epilogue: tcgen05.ld, gates, bfloat16 store; two accumulator
-//             buffers (2 x 256 columns) let it overlap the next tile's MMAs
+//   warps 2-9 epilogue: tcgen05.ld, gates, bfloat16 store (a warp may read only its
+//             own quarter of the 128 lanes, so two warps share a quarter and split
+//             the 64 columns); two accumulator buffers (2 x 256 columns) let the
+//             epilogue overlap the next tile's MMAs
 // Every mbarrier wait is bounded by a wall-clock limit; a wait that runs out
 // raises the block's abort flag, all roles leave their loops, the error word is
 // set and the block still frees its tensor memory.
@@ -47,9 +49,11 @@ constexpr int kBBytes = kBN * kBK * 2;           // 24 KB
 constexpr int kStageBytes = kABytes + kBBytes;   // 40 KB
 constexpr int kAccCols = 4 * kHT;                // one accumulator buffer: nx | r | z | nh
 constexpr int kTmemCols = 2 * kAccCols;          // 512: all of tensor memory
-constexpr int kCellThreads = 192;
+constexpr int kEpilogueWarps = 8;
+constexpr int kCellThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kBarrierBytes = 256;
-constexpr int kCellSmem = kStages * kStageBytes + kBarrierBytes + 1024;  // + slack to align to 1024
+constexpr int kBiasBytes = 4 * GRU_POLICY_MAX_HIDDEN * 4;   // four bias vectors, binary32
+constexpr int kCellSmem = kStages * kStageBytes + kBarrierBytes + kBiasBytes + 1024;  // + slack to align
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait
 constexpr unsigned long long kDrainNs = 200000ull;          // let copies in flight land after an abort
 
@@ -207,15 +211,21 @@ __host__ __device__ constexpr uint32_t instr_desc(int n)
            (static_cast<uint32_t>(kBM >> 4) << 24);
 }
 
-__device__ __forceinline__ float sigmoid_f(float v)
+__device__ __forceinline__ float ex2_approx(float v)
 {
-    return __fdividef(1.0f, 1.0f + __expf(-v));
+    float r;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
 }
 
-__device__ __forceinline__ float tanh_f(float v)
+__device__ __forceinline__ float rcp_approx(float v)
 {
-    return 1.0f - __fdividef(2.0f, __expf(2.0f * v) + 1.0f);
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(v));
+    return r;
 }
+
+constexpr float kLog2e = 1.4426950408889634f;
 
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
@@ -229,8 +239,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 struct CellArgs {
     const __nv_bfloat16 *h_in;
     __nv_bfloat16 *h_out;
-    const float *b_r;   // b_ir + b_hr
-    const float *b_z;   // b_iz + b_hz
+    const float *b_r;   // -log2(e) * (b_ir + b_hr): the sigmoid's exponent is a single fma
+    const float *b_z;   // -log2(e) * (b_iz + b_hz)
     const float *b_in;
     const float *b_hn;
     int n;
@@ -254,6 +264,7 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     const uint32_t acc_full0 = bars + 16 * kStages, acc_empty0 = acc_full0 + 16;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars_ptr + 16 * kStages + 32);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_ptr + 16 * kStages + 40);
+    float *bias_s = reinterpret_cast<float *>(bars_ptr + kBarrierBytes);   // [4][H]: r, z, in, hn
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KC = a.H / kBK;                 // reduction chunks per half
@@ -268,13 +279,19 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full0 + 8 * b, 1);
-            mbar_init(acc_empty0 + 8 * b, 4);   // one arrival per epilogue warp
+            mbar_init(acc_empty0 + 8 * b, kEpilogueWarps);   // one arrival per epilogue warp
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), kTmemCols);
+    for (int i = threadIdx.x; i < a.H; i += kCellThreads) {
+        bias_s[i] = a.b_r[i];
+        bias_s[a.H + i] = a.b_z[i];
+        bias_s[2 * a.H + i] = a.b_in[i];
+        bias_s[3 * a.H + i] = a.b_hn[i];
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -354,6 +371,7 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         }
     } else {
         const int q = warp & 3;                       // the quarter of the lanes this warp may read
+        const int c_begin = ((warp - 2) >> 2) * (kHT / 2);   // and its half of the tile's columns
         const int row_in_tile = q * 32 + lane;
         int it = 0;
         for (int task = blockIdx.x; task < n_tasks; task += gridDim.x, ++it) {
@@ -368,9 +386,8 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
             const size_t off = static_cast<size_t>(live ? row : 0) * a.H + static_cast<size_t>(j) * kHT;
             const uint4 *hrow = reinterpret_cast<const uint4 *>(a.h_in + off);
             uint4 *orow = reinterpret_cast<uint4 *>(a.h_out + off);
-            const int col0 = j * kHT;
 #pragma unroll 1
-            for (int c = 0; c < kHT; c += 16) {
+            for (int c = c_begin; c < c_begin + kHT / 2; c += 16) {
                 uint32_t nx[16], r[16], z[16], nh[16];
                 tmem_ld16(t0 + c, nx);
                 tmem_ld16(t0 + kHT + c, r);
@@ -379,24 +396,33 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
                 uint4 hv[2];
                 hv[0] = live ? __ldg(hrow + c / 8) : make_uint4(0, 0, 0, 0);
                 hv[1] = live ? __ldg(hrow + c / 8 + 1) : make_uint4(0, 0, 0, 0);
+                const float *bs = bias_s + j * kHT + c;
                 tmem_wait_ld();
                 const uint32_t hw[8] = {hv[0].x, hv[0].y, hv[0].z, hv[0].w,
                                         hv[1].x, hv[1].y, hv[1].z, hv[1].w};
                 uint32_t ow[8];
 #pragma unroll
-                for (int i = 0; i < 16; i += 2) {
-                    float o[2];
+                for (int i4 = 0; i4 < 16; i4 += 4) {
+                    const float4 br = *reinterpret_cast<const float4 *>(bs + i4);
+                    const float4 bz = *reinterpret_cast<const float4 *>(bs + a.H + i4);
+                    const float4 bi = *reinterpret_cast<const float4 *>(bs + 2 * a.H + i4);
+                    const float4 bh = *reinterpret_cast<const float4 *>(bs + 3 * a.H + i4);
+                    const float brv[4] = {br.x, br.y, br.z, br.w}, bzv[4] = {bz.x, bz.y, bz.z, bz.w};
+                    const float biv[4] = {bi.x, bi.y, bi.z, bi.w}, bhv[4] = {bh.x, bh.y, bh.z, bh.w};
+                    float o[4];
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int col = col0 + c + i + e;
-                        const float rr = sigmoid_f(__uint_as_float(r[i + e]) + __ldg(a.b_r + col));
-                        const float zz = sigmoid_f(__uint_as_float(z[i + e]) + __ldg(a.b_z + col));
-                        const float cand = tanh_f(__uint_as_float(nx[i + e]) + __ldg(a.b_in + col) +
-                                                  rr * (__uint_as_float(nh[i + e]) + __ldg(a.b_hn + col)));
-                        const float hold = e ? bf16_hi(hw[i / 2]) : bf16_lo(hw[i / 2]);
-                        o[e] = cand + zz * (hold - cand);
+                    for (int e = 0; e < 4; ++e) {
+                        const int i = i4 + e;
+                        // sigmoid(v) = 1 / (1 + 2^(-v log2 e)), tanh(v) = 1 - 2 / (2^(2 v log2 e) + 1)
+                        const float rr = rcp_approx(1.0f + ex2_approx(fmaf(__uint_as_float(r[i]), -kLog2e, brv[e])));
+                        const float zz = rcp_approx(1.0f + ex2_approx(fmaf(__uint_as_float(z[i]), -kLog2e, bzv[e])));
+                        const float pre = fmaf(rr, __uint_as_float(nh[i]) + bhv[e], __uint_as_float(nx[i]) + biv[e]);
+                        const float cand = fmaf(-2.0f, rcp_approx(ex2_approx(pre * (2.0f * kLog2e)) + 1.0f), 1.0f);
+                        const float hold = (i & 1) ? bf16_hi(hw[i / 2]) : bf16_lo(hw[i / 2]);
+                        o[e] = fmaf(zz, hold - cand, cand);
                     }
-                    ow[i / 2] = pack_bf16(o[0], o[1]);
+                    ow[i4 / 2] = pack_bf16(o[0], o[1]);
+                    ow[i4 / 2 + 1] = pack_bf16(o[2], o[3]);
                 }
                 if (live) {
                     orow[c / 8] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
@@ -622,8 +648,8 @@ int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions, 
             }
     std::vector<float> b_r(H), b_z(H), b_in(H), b_hn(H);
     for (int c = 0; c < H; ++c) {
-        b_r[c] = b_ih[c] + b_hh[c];
-        b_z[c] = b_ih[H + c] + b_hh[H + c];
+        b_r[c] = -kLog2e * (b_ih[c] + b_hh[c]);
+        b_z[c] = -kLog2e * (b_ih[H + c] + b_hh[H + c]);
         b_in[c] = b_ih[2 * H + c];
         b_hn[c] = b_hh[2 * H + c];
     }
