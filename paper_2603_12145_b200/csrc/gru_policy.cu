@@ -2,7 +2,7 @@
 // paper's "GRU rollout (~2M parameters)" setting, Table "PufferLib comparisons";
 // Sec. 4, time breakdown) as sm_100a kernels behind the C ABI of gru_policy.h.
 //
-// k_gru_cell is the dense part: per 128-env tile and 64-unit slice of the hidden
+// k_gru_cell is the dense part: per 256-env tile and 64-unit slice of the hidden
 // state it forms the four pre-activation blocks
 //     nx = x W_in^T        r = x W_ir^T + h W_hr^T
 //     nh = h W_hn^T        z = x W_iz^T + h W_hz^T
@@ -15,14 +15,25 @@
 // as [nx | r | z | nh], the x half is one N = 192 instruction into columns 0..191
 // and the h half one N = 192 instruction into columns 64..255, so r and z collect
 // both halves and the two candidate parts stay separate, as the reset gate needs.
+// Every MMA accumulates; the epilogue clears an accumulator buffer after reading it.
+//
+// The kernel runs as clusters of two blocks on the two SMs of a TPC
+// (cta_group::2): each block stages its own 128 rows of x / h and HALF of the
+// weight box (96 rows), the leader block issues M = 256 instructions that read
+// both blocks' shared memory and write both blocks' tensor memory.  A stage is
+// 28 KB per block, so shared memory and L2 see 30 % less traffic per tile than
+// with one block per tile, which is what bounds this shape.
 //
 // Roles in a 320-thread block (one block per SM, persistent over tiles):
-//   warp 0    TMA producer (one lane): fills a 5-deep ring of {x|h tile, weight box}
-//   warp 1    allocates tensor memory; one lane issues the MMAs and commits
-//   warps 2-9 epilogue: tcgen05.ld, gates, bfloat16 store (a warp may read only its
-//             own quarter of the 128 lanes, so two warps share a quarter and split
-//             the 64 columns); two accumulator buffers (2 x 256 columns) let the
-//             epilogue overlap the next tile's MMAs
+//   warp 0    TMA producer (one lane): fills a 7-deep ring of {x|h tile, half weight box};
+//             both blocks' copies complete on the LEADER's full barrier
+//   warp 1    allocates tensor memory; in the leader one lane issues the MMAs and
+//             commits to the empty / accumulator-full barriers of both blocks
+//   warps 2-9 epilogue: tcgen05.ld, gates, bfloat16 store, tcgen05.st of zeros (a warp
+//             may touch only its own quarter of the 128 lanes, so two warps share a
+//             quarter and split the 64 columns); two accumulator buffers (2 x 256
+//             columns) let the epilogue overlap the next tile's MMAs; both blocks'
+//             epilogue warps arrive on the leader's accumulator-empty barrier
 // Every mbarrier wait is bounded by a wall-clock limit; a wait that runs out
 // raises the block's abort flag, all roles leave their loops, the error word is
 // set and the block still frees its tensor memory.
@@ -43,10 +54,11 @@ constexpr int kBM = 128;                         // envs per tile (MMA M)
 constexpr int kBK = 64;                          // reduction elements per stage = one 128-byte row
 constexpr int kHT = 64;                          // hidden units per tile
 constexpr int kBN = 3 * kHT;                     // weight rows per stage (MMA N)
-constexpr int kStages = 5;
-constexpr int kABytes = kBM * kBK * 2;           // 16 KB
-constexpr int kBBytes = kBN * kBK * 2;           // 24 KB
-constexpr int kStageBytes = kABytes + kBBytes;   // 40 KB
+constexpr int kStages = 7;
+constexpr int kABytes = kBM * kBK * 2;           // 16 KB: this block's 128 rows
+constexpr int kBRows = kBN / 2;                  // this block's half of the weight box
+constexpr int kBBytes = kBRows * kBK * 2;        // 12 KB
+constexpr int kStageBytes = kABytes + kBBytes;   // 28 KB per block, 56 KB per pair
 constexpr int kAccCols = 4 * kHT;                // one accumulator buffer: nx | r | z | nh
 constexpr int kTmemCols = 2 * kAccCols;          // 512: all of tensor memory
 constexpr int kEpilogueWarps = 8;
@@ -123,11 +135,37 @@ __device__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_fla
     }
 }
 
+__device__ __forceinline__ uint32_t cluster_cta_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+// The shared::cluster address of this block's shared address `addr` in block `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_rank(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+// Tile load of this block of the pair; `bar` is a shared::cluster address and may be the peer's barrier.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y,
                                             uint32_t bar)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
         " [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
         "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
@@ -145,35 +183,39 @@ __device__ __forceinline__ void tc_fence_after_sync()
 
 __device__ __forceinline__ void tmem_alloc(uint32_t slot, uint32_t cols)
 {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot),
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot),
                  "r"(cols)
                  : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
 
 __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols)
 {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols)
                  : "memory");
 }
 
-// D[tmem] (+)= A[smem] * B[smem]^T, bfloat16 operands, binary32 accumulate.
+// D[tmem] (+)= A[smem] * B[smem]^T over the pair: 256 rows (128 per block), bfloat16
+// operands, binary32 accumulate; each block supplies its rows of A and half of B's rows.
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
                                           uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
         "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 
-// The mbarrier receives one arrival once every MMA issued so far by this thread is done.
-__device__ __forceinline__ void umma_commit(uint32_t bar)
+// The mbarrier at this shared-memory offset in BOTH blocks of the pair receives one
+// arrival once every MMA issued so far by this thread is done.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
-                 : "memory");
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+        "h"(static_cast<uint16_t>(3))
+        : "memory");
 }
 
 // 16 consecutive accumulator columns of this thread's lane.
@@ -194,6 +236,21 @@ __device__ __forceinline__ void tmem_wait_ld()
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Clears 16 consecutive accumulator columns of this thread's lane.
+__device__ __forceinline__ void tmem_zero16(uint32_t taddr)
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
+        "%1, %1, %1, %1};" ::"r"(taddr),
+        "r"(0u)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_wait_st()
+{
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+
 // Shared-memory operand descriptor of a K-major tile whose rows are 128 bytes
 // (64 bfloat16) with the 128-byte swizzle, as TMA writes it: 8-row groups are
 // 1024 bytes apart (stride offset), the leading offset is not used by swizzled
@@ -204,11 +261,12 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr)
            (2ull << 61);
 }
 
-// Instruction descriptor: binary32 accumulator, bfloat16 A and B, both K-major, M = 128.
+// Instruction descriptor: binary32 accumulator, bfloat16 A and B, both K-major,
+// M = 256 across the pair.
 __host__ __device__ constexpr uint32_t instr_desc(int n)
 {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
-           (static_cast<uint32_t>(kBM >> 4) << 24);
+           (static_cast<uint32_t>((2 * kBM) >> 4) << 24);
 }
 
 __device__ __forceinline__ float ex2_approx(float v)
@@ -267,19 +325,21 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     float *bias_s = reinterpret_cast<float *>(bars_ptr + kBarrierBytes);   // [4][H]: r, z, in, hn
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_cta_rank();        // 0 = leader of the pair
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
     const int KC = a.H / kBK;                 // reduction chunks per half
     const int JT = a.H / kHT;                 // hidden tiles
-    const int m_tiles = (a.n + kBM - 1) / kBM;
+    const int m_tiles = (a.n + 2 * kBM - 1) / (2 * kBM);
     const int n_tasks = m_tiles * JT;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full0 + 8 * s, 1);
-            mbar_init(empty0 + 8 * s, 1);
+            mbar_init(full0 + 8 * s, 1);     // the leader's own arrive.expect_tx (used in the leader only)
+            mbar_init(empty0 + 8 * s, 1);    // one commit from the leader's MMA thread
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full0 + 8 * b, 1);
-            mbar_init(acc_empty0 + 8 * b, kEpilogueWarps);   // one arrival per epilogue warp
+            mbar_init(acc_empty0 + 8 * b, 2 * kEpilogueWarps);   // both blocks' epilogue warps (leader only)
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -293,7 +353,7 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         bias_s[3 * a.H + i] = a.b_hn[i];
     }
     tc_fence_before_sync();
-    __syncthreads();
+    cluster_sync_all();          // both blocks' barriers and tensor memory exist from here on
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
 
@@ -301,8 +361,10 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         if (lane == 0) {
             uint32_t s = 0, ph = 0;
             bool ok = true;
-            for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x) {
+            for (int task = pair; task < n_tasks && ok; task += n_pairs) {
                 const int mt = task / JT, j = task - mt * JT;
+                const int row0 = (2 * mt + static_cast<int>(rank)) * kBM;
+                const int wrow0 = j * kBN + static_cast<int>(rank) * kBRows;
                 for (int half = 0; half < 2 && ok; ++half) {
                     const CUtensorMap *ta = half ? &tm_h : &tm_x;
                     const CUtensorMap *tb = half ? &tm_wh : &tm_wx;
@@ -312,9 +374,10 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
                             break;
                         }
                         const uint32_t dst = tiles + s * kStageBytes;
-                        mbar_expect_tx(full0 + 8 * s, kStageBytes);
-                        tma_load_2d(dst, ta, kc * kBK, mt * kBM, full0 + 8 * s);
-                        tma_load_2d(dst + kABytes, tb, kc * kBK, j * kBN, full0 + 8 * s);
+                        const uint32_t leader_full = map_to_rank(full0 + 8 * s, 0);
+                        if (rank == 0) mbar_expect_tx(full0 + 8 * s, 2 * kStageBytes);
+                        tma_load_2d(dst, ta, kc * kBK, row0, leader_full);
+                        tma_load_2d(dst + kABytes, tb, kc * kBK, wrow0, leader_full);
                         if (++s == kStages) {
                             s = 0;
                             ph ^= 1u;
@@ -322,21 +385,28 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
                     }
                 }
             }
+            // do not leave while the leader's MMAs may still read this block's stages
+            for (int i = 0; i < kStages && ok; ++i) {
+                ok = mbar_wait(empty0 + 8 * s, ph ^ 1u, abort_flag);
+                if (++s == kStages) {
+                    s = 0;
+                    ph ^= 1u;
+                }
+            }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t kIdesc192 = instr_desc(kBN);
-            constexpr uint32_t kIdesc128 = instr_desc(2 * kHT);
-            constexpr uint32_t kIdesc64 = instr_desc(kHT);
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t kIdesc = instr_desc(kBN);
             uint32_t s = 0, ph = 0;
             bool ok = true;
             int it = 0;
-            for (int task = blockIdx.x; task < n_tasks && ok; task += gridDim.x, ++it) {
+            for (int task = pair; task < n_tasks && ok; task += n_pairs, ++it) {
                 const uint32_t buf = it & 1, use = (it >> 1) & 1;
-                if (!mbar_wait(acc_empty0 + 8 * buf, use ^ 1u, abort_flag)) break;
+                if (!mbar_wait(acc_empty0 + 8 * buf, use, abort_flag)) break;   // cleared by both epilogues
                 tc_fence_after_sync();
                 const uint32_t d = tmem_base + buf * kAccCols;
                 for (int half = 0; half < 2 && ok; ++half) {
+                    const uint32_t dh = d + (half ? kHT : 0);   // x half: nx|r|z, h half: r|z|nh
                     for (int kc = 0; kc < KC; ++kc) {
                         if (!mbar_wait(full0 + 8 * s, ph, abort_flag)) {
                             ok = false;
@@ -348,41 +418,46 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
 #pragma unroll
                         for (int k = 0; k < kBK / 16; ++k) {
                             // 16 elements = 32 bytes further along the swizzled row: +2 in the address field
-                            const uint64_t ak = ad + 2u * k, bk = bd + 2u * k;
-                            if (half == 0) {
-                                umma_bf16(d, ak, bk, kIdesc192, (kc | k) != 0);
-                            } else if ((kc | k) == 0) {
-                                // first step of the h half: r and z already hold the x half, nh starts here
-                                umma_bf16(d + kHT, ak, bk, kIdesc128, 1u);
-                                umma_bf16(d + 3 * kHT, ak, bk + ((2 * kHT * 128) >> 4), kIdesc64, 0u);
-                            } else {
-                                umma_bf16(d + kHT, ak, bk, kIdesc192, 1u);
-                            }
+                            umma_bf16(dh, ad + 2u * k, bd + 2u * k, kIdesc, 1u);
                         }
-                        umma_commit(empty0 + 8 * s);   // the stage is free once these MMAs have read it
+                        umma_commit_pair(empty0 + 8 * s);   // both blocks' stages are free once these MMAs are done
                         if (++s == kStages) {
                             s = 0;
                             ph ^= 1u;
                         }
                     }
                 }
-                if (ok) umma_commit(acc_full0 + 8 * buf);
+                if (ok) umma_commit_pair(acc_full0 + 8 * buf);
             }
         }
     } else {
-        const int q = warp & 3;                       // the quarter of the lanes this warp may read
+        const int q = warp & 3;                       // the quarter of the lanes this warp may touch
         const int c_begin = ((warp - 2) >> 2) * (kHT / 2);   // and its half of the tile's columns
         const int row_in_tile = q * 32 + lane;
+        const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+        // both accumulator buffers start cleared
+        for (int b = 0; b < 2; ++b) {
+            for (int g = 0; g < 4; ++g)
+                for (int c = c_begin; c < c_begin + kHT / 2; c += 16)
+                    tmem_zero16(lane_base + b * kAccCols + g * kHT + c);
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive_cluster(map_to_rank(acc_empty0, 0));
+            mbar_arrive_cluster(map_to_rank(acc_empty0 + 8, 0));
+        }
         int it = 0;
-        for (int task = blockIdx.x; task < n_tasks; task += gridDim.x, ++it) {
+        for (int task = pair; task < n_tasks; task += n_pairs, ++it) {
             const int mt = task / JT, j = task - mt * JT;
             const uint32_t buf = it & 1, use = (it >> 1) & 1;
             const bool ready = mbar_wait(acc_full0 + 8 * buf, use, abort_flag);
             if (!__all_sync(0xFFFFFFFFu, ready)) break;
             tc_fence_after_sync();
-            const long long row = static_cast<long long>(mt) * kBM + row_in_tile;
+            const long long row = static_cast<long long>(2 * mt + static_cast<int>(rank)) * kBM + row_in_tile;
             const bool live = row < a.n;
-            const uint32_t t0 = tmem_base + buf * kAccCols + (static_cast<uint32_t>(q * 32) << 16);
+            const uint32_t t0 = lane_base + buf * kAccCols;
             const size_t off = static_cast<size_t>(live ? row : 0) * a.H + static_cast<size_t>(j) * kHT;
             const uint4 *hrow = reinterpret_cast<const uint4 *>(a.h_in + off);
             uint4 *orow = reinterpret_cast<uint4 *>(a.h_out + off);
@@ -398,6 +473,10 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
                 hv[1] = live ? __ldg(hrow + c / 8 + 1) : make_uint4(0, 0, 0, 0);
                 const float *bs = bias_s + j * kHT + c;
                 tmem_wait_ld();
+                tmem_zero16(t0 + c);
+                tmem_zero16(t0 + kHT + c);
+                tmem_zero16(t0 + 2 * kHT + c);
+                tmem_zero16(t0 + 3 * kHT + c);
                 const uint32_t hw[8] = {hv[0].x, hv[0].y, hv[0].z, hv[0].w,
                                         hv[1].x, hv[1].y, hv[1].z, hv[1].w};
                 uint32_t ow[8];
@@ -429,9 +508,10 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
                     orow[c / 8 + 1] = make_uint4(ow[4], ow[5], ow[6], ow[7]);
                 }
             }
+            tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty0 + 8 * buf);
+            if (lane == 0) mbar_arrive_cluster(map_to_rank(acc_empty0 + 8 * buf, 0));
         }
     }
 
@@ -442,8 +522,8 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         if (threadIdx.x == 0) atomicExch(a.err, 1);
         const unsigned long long t0 = global_timer_ns();
         while (global_timer_ns() - t0 < kDrainNs) __nanosleep(1000);
-        __syncthreads();
     }
+    cluster_sync_all();          // neither block leaves while its peer may still touch it
     if (warp == 1) {
         __syncwarp();
         tc_fence_after_sync();
@@ -566,6 +646,7 @@ bool encode_operand(TensorMapEncodeFn enc, CUtensorMap *m, const void *base, uin
 struct gru_policy {
     int H = 0, obs_dim = 0, A = 0;
     int device = 0, sms = 0;
+    int pairs = 0;   // clusters of two blocks that can be resident at once
     cudaStream_t stream = nullptr;
     int64_t launches = 0;
     __nv_bfloat16 *wx = nullptr, *wh = nullptr;   // packed [H/64][192][H]
@@ -662,11 +743,28 @@ int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions, 
               upload(&p->err, std::vector<int>(1, 0));
     if (ok) {
         TensorMapEncodeFn enc = tensor_map_encoder();
-        ok = encode_operand(enc, &p->tm_wx, p->wx, H, static_cast<uint64_t>(3) * H, kBN) &&
-             encode_operand(enc, &p->tm_wh, p->wh, H, static_cast<uint64_t>(3) * H, kBN);
+        ok = encode_operand(enc, &p->tm_wx, p->wx, H, static_cast<uint64_t>(3) * H, kBRows) &&
+             encode_operand(enc, &p->tm_wh, p->wh, H, static_cast<uint64_t>(3) * H, kBRows);
     }
     if (ok) ok = cudaFuncSetAttribute(k_gru_cell, cudaFuncAttributeMaxDynamicSharedMemorySize, kCellSmem) ==
                  cudaSuccess;
+    if (ok) {
+        // how many pairs fit on the device at once: the persistent grid is sized to that
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(p->sms & ~1));
+        cfg.blockDim = dim3(kCellThreads);
+        cfg.dynamicSmemBytes = kCellSmem;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int clusters = 0;
+        ok = cudaOccupancyMaxActiveClusters(&clusters, k_gru_cell, &cfg) == cudaSuccess && clusters > 0;
+        p->pairs = clusters < p->sms / 2 ? clusters : p->sms / 2;
+    }
     if (ok && static_cast<size_t>(n_actions) * H * sizeof(float) > 48 * 1024)
         ok = cudaFuncSetAttribute(k_head, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                   static_cast<int>(n_actions * H * sizeof(float))) == cudaSuccess;
@@ -731,10 +829,24 @@ int gru_policy_cell(gru_policy *p, const void *x, const void *h_in, void *h_out,
     a.n = n;
     a.H = p->H;
     a.err = p->err;
-    const long long tasks = static_cast<long long>((n + kBM - 1) / kBM) * (p->H / kHT);
-    const unsigned blocks = static_cast<unsigned>(tasks < p->sms ? tasks : p->sms);
-    k_gru_cell<<<blocks, kCellThreads, kCellSmem, p->stream>>>(tm_x, tm_h, p->tm_wx, p->tm_wh, a);
-    if (cudaGetLastError() != cudaSuccess) return GRU_POLICY_ECUDA;
+    const long long tasks = static_cast<long long>((n + 2 * kBM - 1) / (2 * kBM)) * (p->H / kHT);
+    const long long pairs = tasks < p->pairs ? tasks : p->pairs;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
+    cfg.blockDim = dim3(kCellThreads);
+    cfg.dynamicSmemBytes = kCellSmem;
+    cfg.stream = p->stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, k_gru_cell, tm_x, tm_h, p->tm_wx, p->tm_wh, a) != cudaSuccess) {
+        cudaGetLastError();
+        return GRU_POLICY_ECUDA;
+    }
     p->launches += 1;
     return GRU_POLICY_OK;
 }
