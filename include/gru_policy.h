@@ -56,7 +56,7 @@ extern "C" {
 #define GRU_POLICY_OK        0
 #define GRU_POLICY_EINVAL   (-1)  /* bad size (hidden not a multiple of 64, n < 1, ...) */
 #define GRU_POLICY_ENULL    (-2)  /* required pointer is NULL */
-#define GRU_POLICY_EALIGN   (-3)  /* x / h pointer not 16-byte aligned */
+#define GRU_POLICY_EALIGN   (-3)  /* x / h pointer not 16-byte aligned, obs not 8-byte aligned */
 #define GRU_POLICY_ECUDA    (-4)  /* a CUDA runtime call or launch failed */
 #define GRU_POLICY_ENOMEM   (-5)  /* allocation failed */
 #define GRU_POLICY_ETIMEOUT (-6)  /* a kernel gave up a bounded wait; its output is invalid */
@@ -79,7 +79,7 @@ int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions,
 int gru_policy_destroy(gru_policy *p);
 int gru_policy_set_stream(gru_policy *p, void *cuda_stream);
 
-/* x_out[n][H] (bfloat16) = encoder(obs[n][obs_dim] float32).  If done is not
+/* x_out[n][H] (bfloat16) = encoder(obs[n][obs_dim] float32, 8-byte aligned).  If done is not
  * NULL (uint8[n]) and h is not NULL, row m of h (bfloat16 [n][H]) is set to zero
  * where done[m] != 0: a finished episode starts the next one from a zero state. */
 int gru_policy_encode(gru_policy *p, const float *obs, const uint8_t *done, void *h, void *x_out,

@@ -533,74 +533,146 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
 
 // ---------------------------------------------------------------- encoder and head
 
-// One thread per (env, 8 hidden units): x = bf16(relu(fma chain)), one 16-byte store;
-// also clears the same 8 units of h where the env's episode just ended.
-__global__ void __launch_bounds__(256)
+// Thread t of a block owns hidden units 4t..4t+3 with their encoder weights in
+// registers; the block walks over envs, four per pass.  A warp's stores cover 256
+// contiguous bytes of a row of x.  Where the env's episode just ended the same four
+// units of h are cleared.  OD = obs_dim, known at compile time so that the fma chain
+// is exactly OD long.
+constexpr int kEncodeRows = 4;
+constexpr int kEncodeCols = 4;
+
+template <int OD>
+__global__ void __launch_bounds__(GRU_POLICY_MAX_HIDDEN / kEncodeCols)
 k_encode(const float *__restrict__ obs, const uint8_t *__restrict__ done, __nv_bfloat16 *__restrict__ h,
          __nv_bfloat16 *__restrict__ x_out, const float *__restrict__ enc_w,
-         const float *__restrict__ enc_b, int n, int H, int obs_dim)
+         const float *__restrict__ enc_b, int n, int H)
 {
-    const int groups = H / 8;
-    const long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (idx >= static_cast<long long>(n) * groups) return;
-    const int m = static_cast<int>(idx / groups), g = static_cast<int>(idx - static_cast<long long>(m) * groups);
-    float o[GRU_POLICY_MAX_OBS];
+    const int c = kEncodeCols * threadIdx.x;
+    if (c >= H) return;
+    float w[kEncodeCols][OD], b[kEncodeCols];
 #pragma unroll
-    for (int i = 0; i < GRU_POLICY_MAX_OBS; ++i)
-        o[i] = i < obs_dim ? __ldg(obs + static_cast<size_t>(m) * obs_dim + i) : 0.0f;
-    uint32_t w[4];
+    for (int e = 0; e < kEncodeCols; ++e) {
+        b[e] = __ldg(enc_b + c + e);
 #pragma unroll
-    for (int p = 0; p < 4; ++p) {
-        float v[2];
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-            const int c = g * 8 + 2 * p + e;
-            float acc = __ldg(enc_b + c);
-#pragma unroll
-            for (int i = 0; i < GRU_POLICY_MAX_OBS; ++i)
-                if (i < obs_dim) acc = __fmaf_rn(o[i], __ldg(enc_w + static_cast<size_t>(c) * obs_dim + i), acc);
-            v[e] = acc > 0.0f ? acc : 0.0f;
-        }
-        w[p] = pack_bf16(v[0], v[1]);
+        for (int i = 0; i < OD; ++i) w[e][i] = __ldg(enc_w + static_cast<size_t>(c + e) * OD + i);
     }
-    const size_t off = static_cast<size_t>(m) * H + static_cast<size_t>(g) * 8;
-    *reinterpret_cast<uint4 *>(x_out + off) = make_uint4(w[0], w[1], w[2], w[3]);
-    if (done != nullptr && h != nullptr && __ldg(done + m) != 0)
-        *reinterpret_cast<uint4 *>(h + off) = make_uint4(0, 0, 0, 0);
+    const bool mask = done != nullptr && h != nullptr;
+    for (long long m0 = static_cast<long long>(blockIdx.x) * kEncodeRows; m0 < n;
+         m0 += static_cast<long long>(gridDim.x) * kEncodeRows) {
+        float o[kEncodeRows][OD];
+        bool ended[kEncodeRows];
+#pragma unroll
+        for (int r = 0; r < kEncodeRows; ++r) {
+            const long long m = m0 + r < n ? m0 + r : n - 1;
+            const float *row = obs + static_cast<size_t>(m) * OD;
+            if constexpr (OD % 2 == 0) {   // rows are 8-byte aligned: load pairs
+#pragma unroll
+                for (int i = 0; i < OD; i += 2) {
+                    const float2 v = __ldg(reinterpret_cast<const float2 *>(row + i));
+                    o[r][i] = v.x;
+                    o[r][i + 1] = v.y;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < OD; ++i) o[r][i] = __ldg(row + i);
+            }
+            ended[r] = mask && __ldg(done + m) != 0;
+        }
+#pragma unroll
+        for (int r = 0; r < kEncodeRows; ++r) {
+            if (m0 + r >= n) break;
+            float v[kEncodeCols];
+#pragma unroll
+            for (int e = 0; e < kEncodeCols; ++e) {
+                float acc = b[e];
+#pragma unroll
+                for (int i = 0; i < OD; ++i) acc = __fmaf_rn(o[r][i], w[e][i], acc);
+                v[e] = acc > 0.0f ? acc : 0.0f;
+            }
+            const size_t off = static_cast<size_t>(m0 + r) * H + c;
+            *reinterpret_cast<uint2 *>(x_out + off) = make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
+            if (ended[r]) *reinterpret_cast<uint2 *>(h + off) = make_uint2(0u, 0u);
+        }
+    }
 }
 
-// One thread per env: logits[a] = fma chain over the hidden units in ascending order.
-__global__ void __launch_bounds__(128)
+typedef void (*EncodeKernel)(const float *, const uint8_t *, __nv_bfloat16 *, __nv_bfloat16 *, const float *,
+                             const float *, int, int);
+
+template <int OD>
+struct EncodeTable {
+    static EncodeKernel get(int obs_dim) { return obs_dim == OD ? k_encode<OD> : EncodeTable<OD - 1>::get(obs_dim); }
+};
+template <>
+struct EncodeTable<0> {
+    static EncodeKernel get(int) { return nullptr; }
+};
+
+// 128 envs per block, one thread per env: logits[a] = fma chain over the hidden units
+// in ascending order.  The block brings 64 units of its 128 rows at a time through
+// shared memory with coalesced loads (rows padded to 33 words so that a thread walking
+// its own row meets no bank conflict); the head's weights sit in shared memory as
+// [unit][AP] so that one 16-byte broadcast load feeds up to four chains.
+constexpr int kHeadRows = 128;
+constexpr int kHeadPitch = 33;   // words per staged row: 32 data + 1 pad
+
+template <int AP>   // actions padded to 4 or 8
+__global__ void __launch_bounds__(kHeadRows)
 k_head(const __nv_bfloat16 *__restrict__ h, float *__restrict__ logits, const float *__restrict__ head_w,
        const float *__restrict__ head_b, int n, int H, int A)
 {
-    extern __shared__ float w_s[];   // [A][H]
-    for (int i = threadIdx.x; i < A * H; i += blockDim.x) w_s[i] = head_w[i];
-    __syncthreads();
-    const int m = blockIdx.x * blockDim.x + threadIdx.x;
-    if (m >= n) return;
-    float acc[GRU_POLICY_MAX_ACTIONS];
+    extern __shared__ float4 smem_f4[];
+    float *w_s = reinterpret_cast<float *>(smem_f4);   // [H][AP], then the staged tile
+    uint32_t *tile = reinterpret_cast<uint32_t *>(w_s + AP * H);
+    for (int i = threadIdx.x; i < AP * H; i += kHeadRows) {
+        const int k = i / AP, a = i - k * AP;
+        w_s[i] = a < A ? head_w[static_cast<size_t>(a) * H + k] : 0.0f;
+    }
+    const int m0 = blockIdx.x * kHeadRows;
+    const int m = m0 + threadIdx.x;
+    float acc[AP];
 #pragma unroll
-    for (int a = 0; a < GRU_POLICY_MAX_ACTIONS; ++a) acc[a] = a < A ? __ldg(head_b + a) : 0.0f;
-    const uint4 *row = reinterpret_cast<const uint4 *>(h + static_cast<size_t>(m) * H);
-    for (int k8 = 0; k8 < H / 8; ++k8) {
-        const uint4 v = __ldg(row + k8);
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    for (int a = 0; a < AP; ++a) acc[a] = a < A ? __ldg(head_b + a) : 0.0f;
+    for (int k0 = 0; k0 < H; k0 += 64) {
+        __syncthreads();   // the previous chunk has been read (and, first time, w_s is complete)
 #pragma unroll
-        for (int p = 0; p < 4; ++p) {
-            const float lo = bf16_lo(w[p]), hi = bf16_hi(w[p]);
-            const int k = k8 * 8 + 2 * p;
+        for (int i = 0; i < 8; ++i) {
+            const int piece = i * kHeadRows + threadIdx.x;   // 16-byte pieces, 8 per row
+            const int row = piece >> 3, seg = piece & 7;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (m0 + row < n)
+                v = __ldg(reinterpret_cast<const uint4 *>(h + static_cast<size_t>(m0 + row) * H + k0) + seg);
+            uint32_t *dst = tile + row * kHeadPitch + seg * 4;
+            dst[0] = v.x;
+            dst[1] = v.y;
+            dst[2] = v.z;
+            dst[3] = v.w;
+        }
+        __syncthreads();
+        const uint32_t *mine = tile + threadIdx.x * kHeadPitch;
+        const float4 *wk = reinterpret_cast<const float4 *>(w_s + static_cast<size_t>(k0) * AP);
+#pragma unroll 8
+        for (int p = 0; p < 32; ++p) {
+            const uint32_t word = mine[p];
+            const float hv[2] = {bf16_lo(word), bf16_hi(word)};
 #pragma unroll
-            for (int a = 0; a < GRU_POLICY_MAX_ACTIONS; ++a)
-                if (a < A) {
-                    acc[a] = __fmaf_rn(lo, w_s[a * H + k], acc[a]);
-                    acc[a] = __fmaf_rn(hi, w_s[a * H + k + 1], acc[a]);
+            for (int e = 0; e < 2; ++e) {
+#pragma unroll
+                for (int a4 = 0; a4 < AP / 4; ++a4) {
+                    const float4 wv = wk[(2 * p + e) * (AP / 4) + a4];
+                    acc[4 * a4 + 0] = __fmaf_rn(hv[e], wv.x, acc[4 * a4 + 0]);
+                    acc[4 * a4 + 1] = __fmaf_rn(hv[e], wv.y, acc[4 * a4 + 1]);
+                    acc[4 * a4 + 2] = __fmaf_rn(hv[e], wv.z, acc[4 * a4 + 2]);
+                    acc[4 * a4 + 3] = __fmaf_rn(hv[e], wv.w, acc[4 * a4 + 3]);
                 }
+            }
         }
     }
+    if (m < n) {
 #pragma unroll
-    for (int a = 0; a < GRU_POLICY_MAX_ACTIONS; ++a)
-        if (a < A) logits[static_cast<size_t>(m) * A + a] = acc[a];
+        for (int a = 0; a < AP; ++a)
+            if (a < A) logits[static_cast<size_t>(m) * A + a] = acc[a];
+    }
 }
 
 // ---------------------------------------------------------------- host side
@@ -625,6 +697,12 @@ TensorMapEncodeFn tensor_map_encoder()
         return reinterpret_cast<TensorMapEncodeFn>(p);
     }();
     return fn;
+}
+
+size_t head_smem_bytes(int A, int H)
+{
+    const int AP = A <= 4 ? 4 : 8;
+    return static_cast<size_t>(AP) * H * sizeof(float) + static_cast<size_t>(kHeadRows) * kHeadPitch * 4;
 }
 
 // bfloat16 [rows][H] row-major, boxes of 64 elements x box_rows rows, 128-byte swizzle;
@@ -765,9 +843,10 @@ int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions, 
         ok = cudaOccupancyMaxActiveClusters(&clusters, k_gru_cell, &cfg) == cudaSuccess && clusters > 0;
         p->pairs = clusters < p->sms / 2 ? clusters : p->sms / 2;
     }
-    if (ok && static_cast<size_t>(n_actions) * H * sizeof(float) > 48 * 1024)
-        ok = cudaFuncSetAttribute(k_head, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  static_cast<int>(n_actions * H * sizeof(float))) == cudaSuccess;
+    if (ok && head_smem_bytes(n_actions, H) > 48 * 1024)
+        ok = cudaFuncSetAttribute(n_actions <= 4 ? k_head<4> : k_head<8>,
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  static_cast<int>(head_smem_bytes(n_actions, H))) == cudaSuccess;
     if (!ok) {
         cudaGetLastError();
         release(p);
@@ -797,11 +876,14 @@ int gru_policy_encode(gru_policy *p, const float *obs, const uint8_t *done, void
     if (p == nullptr || obs == nullptr || x_out == nullptr) return GRU_POLICY_ENULL;
     if (n < 1) return GRU_POLICY_EINVAL;
     if ((reinterpret_cast<uintptr_t>(x_out) | reinterpret_cast<uintptr_t>(h)) % 16 != 0) return GRU_POLICY_EALIGN;
-    const long long threads = static_cast<long long>(n) * (p->H / 8);
-    const unsigned blocks = static_cast<unsigned>((threads + 255) / 256);
-    k_encode<<<blocks, 256, 0, p->stream>>>(obs, done, static_cast<__nv_bfloat16 *>(h),
-                                             static_cast<__nv_bfloat16 *>(x_out), p->enc_w, p->enc_b, n,
-                                             p->H, p->obs_dim);
+    if (reinterpret_cast<uintptr_t>(obs) % 8 != 0) return GRU_POLICY_EALIGN;
+    const long long passes = (static_cast<long long>(n) + kEncodeRows - 1) / kEncodeRows;
+    const long long cap = static_cast<long long>(p->sms) * 8;
+    const unsigned blocks = static_cast<unsigned>(passes < cap ? passes : cap);
+    const unsigned threads = static_cast<unsigned>((p->H / kEncodeCols + 31) / 32 * 32);
+    EncodeTable<GRU_POLICY_MAX_OBS>::get(p->obs_dim)<<<blocks, threads, 0, p->stream>>>(
+        obs, done, static_cast<__nv_bfloat16 *>(h), static_cast<__nv_bfloat16 *>(x_out), p->enc_w, p->enc_b, n,
+        p->H);
     if (cudaGetLastError() != cudaSuccess) return GRU_POLICY_ECUDA;
     p->launches += 1;
     return GRU_POLICY_OK;
@@ -856,8 +938,8 @@ int gru_policy_head(gru_policy *p, const void *h, float *logits, int n)
     if (p == nullptr || h == nullptr || logits == nullptr) return GRU_POLICY_ENULL;
     if (n < 1) return GRU_POLICY_EINVAL;
     if (reinterpret_cast<uintptr_t>(h) % 16 != 0) return GRU_POLICY_EALIGN;
-    const unsigned blocks = static_cast<unsigned>((n + 127) / 128);
-    k_head<<<blocks, 128, static_cast<size_t>(p->A) * p->H * sizeof(float), p->stream>>>(
+    const unsigned blocks = static_cast<unsigned>((n + kHeadRows - 1) / kHeadRows);
+    (p->A <= 4 ? k_head<4> : k_head<8>)<<<blocks, kHeadRows, head_smem_bytes(p->A, p->H), p->stream>>>(
         static_cast<const __nv_bfloat16 *>(h), logits, p->head_w, p->head_b, n, p->H, p->A);
     if (cudaGetLastError() != cudaSuccess) return GRU_POLICY_ECUDA;
     p->launches += 1;
