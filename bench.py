@@ -69,10 +69,11 @@ WORKLOADS = {
         env="cartpole", n=1048576, T=32, mode=0, obs_mode=0, frameskip=1, bytes=21.0 + 48.0 / 32,
         kernel="k_cartpole_rollout", traffic=695.4e6),
     "policy65k": dict(
-        name="policy in the loop: GRU policy (2.0 M parameters, bf16, cuBLAS) -> pong_sample_actions -> "
-             "pong_step, N=65536 envs, 32 agent steps per CUDA graph",
+        name="policy in the loop: gru_policy_encode -> gru_policy_cell (tcgen05, 2.0 M parameters, bf16) -> "
+             "gru_policy_head -> pong_sample_actions -> pong_step, N=65536 envs, 32 agent steps per "
+             "CUDA graph",
         env="policy", n=65536, T=32, mode=2, obs_mode=0, frameskip=1, bytes=94.0 + 12.0 + 4.0 + 1.0,
-        kernel="cuBLAS GEMMs (library) + k_sample_actions + k_rollout_vector", traffic=None),
+        kernel="k_gru_cell", traffic=None),
     "small64": dict(
         name="fused vector-obs rollout, N=64 envs, T=2000 steps per launch, in-kernel Philox actions",
         n=64, T=2000, mode=0, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 2000,
@@ -229,10 +230,12 @@ def run_reference(args, rank):
 def run_policy(args, w, rank, world, local):
     """The policy-in-the-loop workload: K agent steps per CUDA graph replay; a
     "step" of the benchmark is one replay.  Also times the same graph without the
-    env-side kernels to report the env's share of the step."""
+    env-side kernels, and the cell kernel alone, to report each part's share."""
     import torch
-    from paper_2603_12145_b200 import policy_loop, pong, sharding
+    from paper_2603_12145_b200 import gru_policy, policy_loop, pong, sharding
+    from paper_2603_12145_b200.inputs import policy_weights
     import oracle
+    from oracle import gru_policy as ogp
     import numpy as np
 
     N, K = w["n"], w["T"]
@@ -240,8 +243,10 @@ def run_policy(args, w, rank, world, local):
     steps = args.steps if args.steps > 0 else 100
     warmup = max(args.warmup, 3)
     env_id_base, _ = sharding.shard(rank, world, N)
-    policy = policy_loop.make_policy(hidden=hidden, seed=SEED, dtype=torch.bfloat16)
-    n_params = sum(p.numel() for p in policy.parameters())
+    gru_policy.load(build_if_missing=True)
+    params = policy_weights(hidden, SEED)
+    policy = gru_policy.GruPolicy(params, device="cuda:%d" % local)
+    n_params = sum(int(np.asarray(v).size) for v in params.values())
 
     def timed(with_env, with_policy=True):
         loop = policy_loop.PolicyLoop(pong.PongEnv(N, SEED, env_id_base=env_id_base), policy, K)
@@ -249,7 +254,7 @@ def run_policy(args, w, rank, world, local):
         for _ in range(warmup):
             loop.replay()
         torch.cuda.synchronize()
-        l0 = loop.env.launches
+        l0 = loop.env.launches + policy.launches
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         w0 = time.perf_counter()
         e0.record()
@@ -257,71 +262,91 @@ def run_policy(args, w, rank, world, local):
             loop.replay()
         e1.record()
         torch.cuda.synchronize()
-        return e0.elapsed_time(e1), w0, time.perf_counter(), loop, loop.env.launches - l0
+        # launches made while capturing are replayed: count kernels per replay from what a step launches
+        per_replay = K * ((3 if with_policy else 0) + (2 if with_env else 0)) + (1 if with_env else 0)
+        return e0.elapsed_time(e1), w0, time.perf_counter(), loop, steps * per_replay + 0 * l0
 
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
-    ms_env, w0, w1, loop, fill_launches = timed(True)
+    ms_env, w0, w1, loop, launches = timed(True)
     ms_pol, _, _, _, _ = timed(False)
     ms_envk, _, _, _, _ = timed(True, with_policy=False)
-    # end to end: the step's metric (summed reward) is read back to the host after every replay
+    # the cell kernel alone, back to back, on the loop's own buffers
+    policy._stream()
+    cell_reps = K * min(steps, 20)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(3):
+        gru_policy.gru_policy_cell(policy.h, loop.x, loop.h[0], loop.h[1], N)
+    e0.record()
+    for _ in range(cell_reps):
+        gru_policy.gru_policy_cell(policy.h, loop.x, loop.h[0], loop.h[1], N)
+    e1.record()
+    torch.cuda.synchronize()
+    cell_ms = e0.elapsed_time(e1) / cell_reps
+    policy.status()
+    # end to end: the step's result (the env's episode statistics) is read back after every replay
     e2e_steps = max(args.e2e_steps, 1)
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         loop.replay()
-        float(loop.reward_sum.item())
+        stats = loop.env.episode_stats()
     e2e_s = time.perf_counter() - t0
     sampler.stop()
     ms_env = sharding.max_over_ranks(ms_env, device="cuda")
     value = world * steps * N * K / (ms_env * 1e-3)
-    flops = 2.0 * n_params * N * K * steps
+    cell_flops = 2.0 * 6 * hidden * hidden * N          # the six H x H products of one agent step
     try:
-        peak_tf = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
-        peak_kind = "measured"
+        peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
+        peak_tf, peak_kind = float(peaks["bf16_tflops_sustained"]), "measured, sustained"
     except Exception:
-        peak_tf, peak_kind = 1590.0, "fallback"
-    achieved_tf = flops / (ms_env * 1e-3) / 1e12
+        peak_tf, peak_kind = 1400.0, "fallback, sustained"
+    achieved_tf = cell_flops / (cell_ms * 1e-3) / 1e12
     if rank != 0:
         return
-    # CPU: the env-side part only (sampling from given logits + env step); the policy
-    # network has no oracle, it is a library call
-    n_s = 8192
+    # CPU: the whole agent step from the oracles (encoder, binary64 cell, head, sampling, env step)
+    n_s = 256
     o = oracle.OraclePong(n_s, SEED)
-    rng = np.random.Generator(np.random.PCG64(SEED))
-    logits = rng.normal(0, 1, (n_s, 3)).astype(np.float32)
+    obs = o.reset()
+    h = np.zeros((n_s, hidden), np.float32)
     c0, reps = time.perf_counter(), 0
     while time.perf_counter() - c0 < max(args.cpu_seconds, 0.2):
-        words = o.fill_words(K)
-        for i in range(K):
-            o.step(oracle.sample_actions(logits, words[i]))
+        words = o.fill_words(1)
+        x = ogp.encode(obs, params["enc_w"], params["enc_b"])
+        h = ogp.bf16_round_f64(ogp.cell(x, h, params["w_ih"], params["w_hh"], params["b_ih"], params["b_hh"]))
+        logits = ogp.head(h, params["head_w"], params["head_b"])
+        obs, _, done = o.step(oracle.sample_actions(logits, words[0]))
+        h[done != 0] = 0.0
         reps += 1
     cpu_dt = time.perf_counter() - c0
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": ms_env / steps, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16 policy, int32 env", "data": "synthetic",
+        "vs_baseline": None, "dtype": "bf16 policy (f32 accumulate), int32 env", "data": "synthetic",
         "config": {"workload": w["name"], "workload_key": args.workload, "n_envs_per_gpu": N,
                    "agent_steps_per_graph": K, "policy_parameters": n_params, "hidden": hidden,
                    "env_steps_per_step": N * K,
-                   "l2": "the policy's activations and weights are read every step; no flush"},
+                   "l2": "the policy's activations (226 MB) and weights are read every step; no flush"},
         "roofline": {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
                      "frac": achieved_tf / peak_tf, "peak_source": peak_kind + " cuBLAS bf16",
-                     "traffic": None, "kernel": w["kernel"],
-                     "note": "the matrix products are cuBLAS library calls made by torch; 2 x parameters "
-                             "x envs flops per agent step"},
-        "policy_only_ms_per_step": ms_pol / steps,
-        "env_kernels_only_ms_per_step": ms_envk / steps,
+                     "traffic": None, "kernel": w["kernel"], "kernel_ms": cell_ms,
+                     "flops_per_launch": cell_flops,
+                     "note": "12 H^2 flops per env: the six H x H products of the GRU cell, timed back "
+                             "to back on the loop's buffers"},
+        "agent_step_us": ms_env / steps / K * 1e3,
+        "policy_only_us_per_agent_step": ms_pol / steps / K * 1e3,
+        "env_kernels_only_us_per_agent_step": ms_envk / steps / K * 1e3,
+        "cell_kernel_us": cell_ms * 1e3,
         "env_kernels_share_of_step": ms_envk / ms_env,
-        "env_and_bookkeeping_share_of_step": (ms_env - ms_pol) / ms_env,
         "e2e": {"value": world * e2e_steps * N * K / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 0,
-                "d2h_bytes_per_step": 8, "steps": e2e_steps,
-                "api": "PolicyLoop.replay + read-back of the summed reward"},
-        "gpu_launches": int(fill_launches + steps * K * 2),
+                "d2h_bytes_per_step": 24, "steps": e2e_steps,
+                "api": "PolicyLoop.replay + read-back of the env's episode statistics"},
+        "gpu_launches": int(launches),
         "clocks": sampler.summary(w0, w1),
-        "cpu_baseline": {"value": reps * n_s * K / cpu_dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+        "episode_stats": dict(zip(("episodes", "sum_return", "sum_length"), (int(v) for v in stats))),
+        "cpu_baseline": {"value": reps * n_s / cpu_dt, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "host_cores": os.cpu_count(),
-                         "sample": "env-side part only (sampling from fixed logits + env step), envs "
-                                   "0..8191, %d x %d steps, %.1f s, single thread" % (reps, K, cpu_dt)},
+                         "sample": "whole agent step (encoder, binary64 cell, head, sampling, env step) "
+                                   "of envs 0..%d, %d steps, %.1f s, single thread" % (n_s - 1, reps, cpu_dt)},
     }
     print(json.dumps(line), flush=True)
 

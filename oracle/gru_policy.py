@@ -37,6 +37,8 @@ def lib():
             vp, i32, f32 = ctypes.c_void_p, ctypes.c_int, ctypes.c_float
             L.gp_oracle_bf16_round.argtypes = [f32]
             L.gp_oracle_bf16_round.restype = f32
+            L.gp_oracle_bf16_round_f64.argtypes = [vp, vp, ctypes.c_size_t]
+            L.gp_oracle_bf16_round_f64.restype = None
             L.gp_oracle_encode.argtypes = [vp, i32, i32, i32, vp, vp, vp]
             L.gp_oracle_encode.restype = None
             L.gp_oracle_cell.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp, vp]
@@ -53,6 +55,14 @@ def _f32(a):
 
 def bf16_round(v: float) -> float:
     return float(lib().gp_oracle_bf16_round(float(np.float32(v))))
+
+
+def bf16_round_f64(a) -> np.ndarray:
+    """float32 array of the bfloat16 values nearest to the float64 array a."""
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    out = np.empty(a.shape, dtype=np.float32)
+    lib().gp_oracle_bf16_round_f64(a.ctypes.data, out.ctypes.data, a.size)
+    return out
 
 
 def encode(obs, enc_w, enc_b) -> np.ndarray:

@@ -41,6 +41,7 @@
  * bit patterns and ties.
  */
 #include <math.h>
+#include <stddef.h>
 #include <stdint.h>
 #include <string.h>
 
@@ -61,6 +62,26 @@ float gp_oracle_bf16_round(float v)
     float r;
     memcpy(&r, &u, 4);
     return r;
+}
+
+/* out[i] = bfloat16 nearest to the binary64 in[i] (ties to even), as a binary32.
+ * One rounding: the binary64 is first cut to binary32 toward zero with a sticky
+ * last bit (round to odd), which the final rounding to 8 significant bits cannot
+ * tell from the exact value. */
+void gp_oracle_bf16_round_f64(const double *in, float *out, size_t count)
+{
+    for (size_t i = 0; i < count; ++i) {
+        double d = in[i];
+        float f = (float)d;
+        if (f == f && f - f == 0.0f && (double)f != d) {   /* finite and inexact */
+            if (fabs((double)f) > fabs(d)) f = nextafterf(f, 0.0f);
+            uint32_t u;
+            memcpy(&u, &f, 4);
+            u |= 1u;
+            memcpy(&f, &u, 4);
+        }
+        out[i] = gp_oracle_bf16_round(f);
+    }
 }
 
 /* x[n][H] = bf16(relu(b_e[c] + sum_i obs[i] * W_e[c][i])), binary32 fma chain, i ascending */

@@ -80,3 +80,21 @@ def test_cartpole_library_exports_every_declared_symbol():
     assert L.cartpole_create(ctypes.byref(h), 0, 0, 0) == -1
     assert L.cartpole_create(ctypes.byref(h), 4, 0, -1) == -1
     assert L.cartpole_create(None, 4, 0, 0) == -2
+
+
+def test_gru_policy_library_exports_every_declared_symbol():
+    from paper_2603_12145_b200 import gru_policy
+    lib = ctypes.CDLL(build.build_one("libgru_policy_b200.so"))
+    names = declared_symbols("gru_policy.h", "gru_policy")
+    assert len(names) >= 10
+    for name in names:
+        assert hasattr(lib, name), name
+    assert set(names) == set(gru_policy.EXPORTS)
+    L = gru_policy.load(build_if_missing=True)
+    assert gru_policy.strerror(0) == "ok" and gru_policy.strerror(-6).startswith("a kernel gave up")
+    # argument checks that run before any CUDA call
+    assert L.gru_policy_create(None, 64, 6, 3, *([None] * 8)) == -2
+    h = ctypes.c_void_p()
+    assert L.gru_policy_create(ctypes.byref(h), 64, 6, 3, *([None] * 8)) == -2
+    assert L.gru_policy_destroy(None) == -2 and L.gru_policy_status(None) == -2
+    assert L.gru_policy_cell(None, None, None, None, 1) == -2

@@ -39,6 +39,20 @@ def test_bf16_rounding_against_torch():
     assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
 
 
+def test_bf16_rounding_of_float64_is_a_single_rounding():
+    # 1 + 2^-8 is a tie (-> 1.0); the same plus 2^-40 lies above the tie, but rounding it to
+    # binary32 first would land back on the tie: a double rounding would return 1.0
+    v = np.array([1.0 + 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -40, 1.0 + 2.0 ** -8 - 2.0 ** -40,
+                  -(1.0 + 3 * 2.0 ** -8 - 2.0 ** -40), 0.0, 1e-3, -2.5])
+    want = np.array([1.0, 1.0 + 2.0 ** -7, 1.0, -(1.0 + 2.0 ** -7), 0.0,
+                     gp.bf16_round(1e-3), -2.5], dtype=np.float32)
+    assert np.array_equal(gp.bf16_round_f64(v), want)
+    rng = np.random.Generator(np.random.PCG64(6))
+    f = rng.normal(0, 1, 2000).astype(np.float32)
+    assert np.array_equal(gp.bf16_round_f64(f.astype(np.float64)),
+                          np.array([gp.bf16_round(x) for x in f], dtype=np.float32))
+
+
 @pytest.mark.parametrize("H,n,seed", [(64, 5, 1), (192, 3, 2)])
 def test_cell_against_torch_grucell_float64(H, n, seed):
     import torch
