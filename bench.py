@@ -248,13 +248,15 @@ def run_policy(args, w, rank, world, local):
     policy = gru_policy.GruPolicy(params, device="cuda:%d" % local)
     n_params = sum(int(np.asarray(v).size) for v in params.values())
 
+    parts = max(1, args.parts)
+
     def timed(with_env, with_policy=True):
-        loop = policy_loop.PolicyLoop(pong.PongEnv(N, SEED, env_id_base=env_id_base), policy, K)
+        loop = policy_loop.PipelinedPolicyLoop(N, SEED, policy, K, parts=parts, env_id_base=env_id_base,
+                                               device="cuda:%d" % local)
         loop.capture(with_env=with_env, with_policy=with_policy)
         for _ in range(warmup):
             loop.replay()
         torch.cuda.synchronize()
-        l0 = loop.env.launches + policy.launches
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         w0 = time.perf_counter()
         e0.record()
@@ -263,23 +265,27 @@ def run_policy(args, w, rank, world, local):
         e1.record()
         torch.cuda.synchronize()
         # launches made while capturing are replayed: count kernels per replay from what a step launches
-        per_replay = K * ((3 if with_policy else 0) + (2 if with_env else 0)) + (1 if with_env else 0)
-        return e0.elapsed_time(e1), w0, time.perf_counter(), loop, steps * per_replay + 0 * l0
+        per_replay = parts * (K * ((3 if with_policy else 0) + (2 if with_env else 0)) + (1 if with_env else 0))
+        return e0.elapsed_time(e1), w0, time.perf_counter(), loop, steps * per_replay
 
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
     ms_env, w0, w1, loop, launches = timed(True)
     ms_pol, _, _, _, _ = timed(False)
     ms_envk, _, _, _, _ = timed(True, with_policy=False)
-    # the cell kernel alone, back to back, on the loop's own buffers
+    # the cell kernel alone, back to back, all N envs per launch, on operands of the loop's kind
     policy._stream()
+    gen = torch.Generator(device="cuda:%d" % local).manual_seed(SEED)
+    cx = torch.rand((N, hidden), device="cuda:%d" % local, generator=gen).to(torch.bfloat16)
+    ch = (torch.rand((N, hidden), device="cuda:%d" % local, generator=gen) * 2 - 1).to(torch.bfloat16)
+    cout = torch.empty_like(ch)
     cell_reps = K * min(steps, 20)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for _ in range(3):
-        gru_policy.gru_policy_cell(policy.h, loop.x, loop.h[0], loop.h[1], N)
+        gru_policy.gru_policy_cell(policy.h, cx, ch, cout, N)
     e0.record()
     for _ in range(cell_reps):
-        gru_policy.gru_policy_cell(policy.h, loop.x, loop.h[0], loop.h[1], N)
+        gru_policy.gru_policy_cell(policy.h, cx, ch, cout, N)
     e1.record()
     torch.cuda.synchronize()
     cell_ms = e0.elapsed_time(e1) / cell_reps
@@ -289,7 +295,7 @@ def run_policy(args, w, rank, world, local):
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
         loop.replay()
-        stats = loop.env.episode_stats()
+        stats = loop.episode_stats()
     e2e_s = time.perf_counter() - t0
     sampler.stop()
     ms_env = sharding.max_over_ranks(ms_env, device="cuda")
@@ -324,6 +330,7 @@ def run_policy(args, w, rank, world, local):
         "vs_baseline": None, "dtype": "bf16 policy (f32 accumulate), int32 env", "data": "synthetic",
         "config": {"workload": w["name"], "workload_key": args.workload, "n_envs_per_gpu": N,
                    "agent_steps_per_graph": K, "policy_parameters": n_params, "hidden": hidden,
+                   "parallel_slices": parts,
                    "env_steps_per_step": N * K,
                    "l2": "the policy's activations (226 MB) and weights are read every step; no flush"},
         "roofline": {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
@@ -331,7 +338,7 @@ def run_policy(args, w, rank, world, local):
                      "traffic": None, "kernel": w["kernel"], "kernel_ms": cell_ms,
                      "flops_per_launch": cell_flops,
                      "note": "12 H^2 flops per env: the six H x H products of the GRU cell, timed back "
-                             "to back on the loop's buffers"},
+                             "to back over all N envs"},
         "agent_step_us": ms_env / steps / K * 1e3,
         "policy_only_us_per_agent_step": ms_pol / steps / K * 1e3,
         "env_kernels_only_us_per_agent_step": ms_envk / steps / K * 1e3,
@@ -360,6 +367,8 @@ def main():
     ap.add_argument("--workload", default="rollout65k", choices=sorted(WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--parts", type=int, default=2,
+                    help="policy65k: independent env slices run as parallel chains of one graph")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))

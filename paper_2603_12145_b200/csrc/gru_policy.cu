@@ -725,6 +725,7 @@ struct gru_policy {
     int H = 0, obs_dim = 0, A = 0;
     int device = 0, sms = 0;
     int pairs = 0;   // clusters of two blocks that can be resident at once
+    int top_priority = 0;   // numerically lowest = most urgent launch priority of the device
     cudaStream_t stream = nullptr;
     int64_t launches = 0;
     __nv_bfloat16 *wx = nullptr, *wh = nullptr;   // packed [H/64][192][H]
@@ -788,6 +789,11 @@ int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions, 
         return GRU_POLICY_ECUDA;
     }
     p->sms = prop.multiProcessorCount;
+    int least = 0;
+    if (cudaDeviceGetStreamPriorityRange(&least, &p->top_priority) != cudaSuccess) {
+        cudaGetLastError();
+        p->top_priority = 0;
+    }
 
     // Pack the weights: tile j holds, for the x half, rows [W_in | W_ir | W_iz] of its 64 units
     // and, for the h half, rows [W_hr | W_hz | W_hn]; gate blocks of the inputs are r, z, n.
@@ -826,6 +832,10 @@ int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions, 
     }
     if (ok) ok = cudaFuncSetAttribute(k_gru_cell, cudaFuncAttributeMaxDynamicSharedMemorySize, kCellSmem) ==
                  cudaSuccess;
+    // Ask for the largest shared-memory partition, not the smallest that holds one block, so that
+    // small blocks of other kernels can share an SM with a cell block.
+    if (ok) ok = cudaFuncSetAttribute(k_gru_cell, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                      cudaSharedmemCarveoutMaxShared) == cudaSuccess;
     if (ok) {
         // how many pairs fit on the device at once: the persistent grid is sized to that
         cudaLaunchConfig_t cfg = {};
@@ -918,13 +928,17 @@ int gru_policy_cell(gru_policy *p, const void *x, const void *h_in, void *h_out,
     cfg.blockDim = dim3(kCellThreads);
     cfg.dynamicSmemBytes = kCellSmem;
     cfg.stream = p->stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // The cell wants whole SMs; when it is pending together with small kernels of a parallel
+    // chain, its blocks are placed first and the small kernels take what is left.
+    attr[1].id = cudaLaunchAttributePriority;
+    attr[1].val.priority = p->top_priority;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (cudaLaunchKernelEx(&cfg, k_gru_cell, tm_x, tm_h, p->tm_wx, p->tm_wh, a) != cudaSuccess) {
         cudaGetLastError();
         return GRU_POLICY_ECUDA;

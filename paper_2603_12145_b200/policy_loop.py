@@ -116,3 +116,85 @@ class PolicyLoop:
         self.graph.replay()
         if self.with_env:
             self.env.t = self.env.t + self.K
+
+
+class PipelinedPolicyLoop:
+    """The same loop over `parts` disjoint slices of the envs, each slice a
+    PolicyLoop of its own on its own stream, all captured into one CUDA graph.
+
+    The slices are independent (envs are), so the graph has `parts` parallel
+    chains and the device overlaps one slice's small memory-bound kernels
+    (encoder, head, sampling, env step) with another slice's tensor-core cell.
+    Env ids are global (`env_id_base` + slice offset): the union of the slices'
+    trajectories is the trajectory of one loop over all envs."""
+
+    def __init__(self, n_envs: int, seed: int, policy: "gru_policy.GruPolicy", steps_per_graph: int = 32,
+                 parts: int = 2, env_id_base: int = 0, device=None):
+        import torch
+        if parts < 1 or n_envs % parts:
+            raise ValueError("n_envs must be a multiple of parts")
+        self.torch, self.policy, self.K, self.n = torch, policy, int(steps_per_graph), int(n_envs)
+        per = n_envs // parts
+        dev = str(device) if device is not None else str(policy.device)
+        self.parts = [PolicyLoop(pong.PongEnv(per, seed, env_id_base=env_id_base + i * per, device=dev),
+                                 policy, steps_per_graph) for i in range(parts)]
+        self.device = self.parts[0].env.device
+        self.streams = [torch.cuda.Stream(device=self.device) for _ in self.parts]
+        self.graph = None
+        self.with_env = True
+
+    def run_eager(self, steps: int):
+        for part in self.parts:
+            part.run_eager(steps)
+
+    def capture(self, with_env: bool = True, with_policy: bool = True):
+        t = self.torch
+        t0 = [part.env.t for part in self.parts]
+        side = t.cuda.Stream(device=self.device)
+        side.wait_stream(t.cuda.current_stream(self.device))
+        with t.cuda.stream(side):
+            scratch = PolicyLoop(pong.PongEnv(64, 0, device=str(self.device)), self.policy, 2)
+            scratch.run_eager(2)
+            self.policy.status()
+            scratch.env.close()
+        t.cuda.current_stream(self.device).wait_stream(side)
+        self.graph = t.cuda.CUDAGraph()
+        with t.cuda.graph(self.graph):
+            main = t.cuda.current_stream(self.device)
+            for part, stream in zip(self.parts, self.streams):
+                stream.wait_stream(main)
+            # issue the chains step by step in turn, so that the capture order (which the
+            # device's scheduler tends to follow) already interleaves them
+            for i in range(self.K):
+                for part, stream in zip(self.parts, self.streams):
+                    with t.cuda.stream(stream):
+                        part._streams()
+                        part._step(i, with_env, with_policy)
+            for stream in self.streams:
+                main.wait_stream(stream)
+        for part, start in zip(self.parts, t0):
+            part._streams()
+            part.env.t = start
+        self.with_env = with_env
+
+    def replay(self):
+        if self.with_env:
+            for part in self.parts:
+                part._streams()
+                pong.pong_fill_words(part.env.h, self.K, part.words)
+        self.graph.replay()
+        if self.with_env:
+            for part in self.parts:
+                part.env.t = part.env.t + self.K
+
+    def episode_stats(self):
+        totals = [0, 0, 0]
+        for part in self.parts:
+            part._streams()
+            for i, v in enumerate(part.env.episode_stats()):
+                totals[i] += int(v)
+        return tuple(totals)
+
+    @property
+    def launches(self) -> int:
+        return sum(part.env.launches for part in self.parts)

@@ -148,3 +148,28 @@ def test_loop_against_an_independent_oracle_loop(torch):
     assert worst_h <= 2.0 ** -6, worst_h          # a few places of 2^-8 relative at |h| <= 1
     assert worst_margin <= 2e-3, worst_margin
     assert (~same).mean() <= 0.02, (~same).sum()
+
+
+def test_pipelined_loop_equals_the_single_loop(torch):
+    """Two slices on two streams in one graph: the union of their trajectories is the
+    single loop's, bit for bit (global env ids; the cell's result for a row does not
+    depend on where the row sits in a tile)."""
+    n, seed, K, H = 1024, 4, 6, 128
+    pol = gru_policy.GruPolicy(policy_weights(H, 3))
+    one = policy_loop.PolicyLoop(pong.PongEnv(n, seed), pol, steps_per_graph=K)
+    two = policy_loop.PipelinedPolicyLoop(n, seed, pol, steps_per_graph=K, parts=2)
+    two.capture()
+    for rep in range(4):
+        one.run_eager(K)
+        two.replay()
+        torch.cuda.synchronize()
+        for name in ("obs", "actions", "done", "logits", "reward"):
+            whole = getattr(one, name)
+            halves = torch.cat([getattr(p, name) for p in two.parts])
+            assert torch.equal(whole, halves), name
+        assert torch.equal(one.hidden, torch.cat([p.hidden for p in two.parts]))
+    assert two.episode_stats() == tuple(int(v) for v in one.env.episode_stats())
+    states = [p.env.get_state() for p in two.parts]
+    assert np.array_equal(np.concatenate([s[0] for s in states], axis=1), one.env.get_state()[0])
+    assert all(s[1] == one.env.get_state()[1] for s in states)
+    pol.status()
