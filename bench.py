@@ -367,7 +367,7 @@ def main():
     ap.add_argument("--workload", default="rollout65k", choices=sorted(WORKLOADS))
     ap.add_argument("--e2e-steps", type=int, default=8)
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
-    ap.add_argument("--parts", type=int, default=2,
+    ap.add_argument("--parts", type=int, default=1,
                     help="policy65k: independent env slices run as parallel chains of one graph")
     args = ap.parse_args()
 

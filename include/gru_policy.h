@@ -30,10 +30,13 @@
  *    tensor cores is not specified, so h' is defined up to that: it agrees with
  *    an exact evaluation to within one bfloat16 rounding plus a binary32
  *    accumulation error (see the parity tests for the bound).
- *  - gru_policy_head: binary32, one fused multiply-add per hidden unit starting
- *    from the bias, units in ascending order.  Reproducible bit for bit, so an
- *    action sampled from these logits is decided identically by any
- *    implementation that follows the same order.
+ *  - gru_policy_head: binary32.  The hidden units are taken in blocks of 32; a
+ *    block's partial sum is a chain of fused multiply-adds from zero over its
+ *    units in ascending order; the logit is the bias plus the partial sums added
+ *    one by one in block order.  Reproducible bit for bit, so an action sampled
+ *    from these logits is decided identically by any implementation that follows
+ *    the same order.  gru_policy_cell_head forms the partial sums in the cell's
+ *    epilogue, where each block of h' is produced, and gives the same bits.
  *
  * Conventions.  Parameters are given to gru_policy_create as HOST float arrays,
  * rows = output units, gate blocks of w_ih / w_hh / b_ih / b_hh in the order
@@ -47,6 +50,7 @@
 #ifndef GRU_POLICY_H_
 #define GRU_POLICY_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -91,6 +95,17 @@ int gru_policy_cell(gru_policy *p, const void *x, const void *h_in, void *h_out,
 
 /* logits[n][n_actions] (float32) = head(h[n][H] bfloat16). */
 int gru_policy_head(gru_policy *p, const void *h, float *logits, int n);
+
+/* Bytes of device scratch gru_policy_cell_head needs for n envs (0 if p is NULL or n < 1). */
+size_t gru_policy_workspace_bytes(const gru_policy *p, int n);
+
+/* gru_policy_cell followed by gru_policy_head on its result, with the head's partial
+ * sums formed inside the cell kernel: h_out as gru_policy_cell, logits as
+ * gru_policy_head(h_out).  workspace: device scratch of gru_policy_workspace_bytes(p, n)
+ * bytes, 16-byte aligned, owned by the caller.  Needs n_actions <= 4 and hidden <= 896
+ * (GRU_POLICY_EINVAL otherwise: call the two entry points separately). */
+int gru_policy_cell_head(gru_policy *p, const void *x, const void *h_in, void *h_out, float *logits,
+                         void *workspace, int n);
 
 /* Synchronises the stream; GRU_POLICY_ETIMEOUT if any kernel since the last call
  * gave up a wait (clears the flag), GRU_POLICY_ECUDA on a CUDA error, else 0. */

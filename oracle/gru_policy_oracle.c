@@ -27,9 +27,13 @@
  *    bound scales with.
  *  - The encoder output is rounded to bfloat16 (it is a tensor-core operand)
  *    and the head's logits decide the sampled action, so both are written in
- *    binary32 with one fixed order: a chain of fused multiply-adds starting
- *    from the bias, k ascending.  fmaf is correctly rounded, so a second
- *    implementation can reproduce every bit.
+ *    binary32 with one fixed order: the encoder as a chain of fused
+ *    multiply-adds starting from the bias, inputs ascending; the head as such
+ *    chains over blocks of 32 hidden units, each from zero, whose results are
+ *    added to the bias in block order (the block structure lets a device
+ *    produce a block's partial sum where the block of hidden units is made).
+ *    fmaf and + are correctly rounded, so a second implementation can
+ *    reproduce every bit.
  *  - bfloat16 rounding is round-to-nearest-even on the upper 16 bits.
  *
  * One row (env) at a time, plain loops; shares no code with the CUDA path.
@@ -138,16 +142,24 @@ void gp_oracle_cell(const float *x, const float *h, int n, int H, const float *w
     }
 }
 
-/* logits[n][A] = b_o[a] + sum_k h[k] * W_o[a][k], binary32 fma chain, k ascending */
+/* logits[n][A]: the hidden units are taken in blocks of 32; a block's partial sum is a
+ * binary32 fma chain from zero over its units in ascending order; the logit is the bias
+ * plus the partial sums, added one by one in block order. */
+enum { GP_HEAD_BLOCK = 32 };
+
 void gp_oracle_head(const float *h, int n, int H, int A, const float *head_w, const float *head_b,
                     float *logits)
 {
     for (int m = 0; m < n; ++m) {
         for (int a = 0; a < A; ++a) {
-            float acc = head_b[a];
-            for (int k = 0; k < H; ++k)
-                acc = fmaf(h[(size_t)m * H + k], head_w[(size_t)a * H + k], acc);
-            logits[(size_t)m * A + a] = acc;
+            float total = head_b[a];
+            for (int k0 = 0; k0 < H; k0 += GP_HEAD_BLOCK) {
+                float part = 0.0f;
+                for (int k = k0; k < k0 + GP_HEAD_BLOCK && k < H; ++k)
+                    part = fmaf(h[(size_t)m * H + k], head_w[(size_t)a * H + k], part);
+                total = total + part;
+            }
+            logits[(size_t)m * A + a] = total;
         }
     }
 }

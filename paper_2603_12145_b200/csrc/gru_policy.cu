@@ -64,8 +64,13 @@ constexpr int kTmemCols = 2 * kAccCols;          // 512: all of tensor memory
 constexpr int kEpilogueWarps = 8;
 constexpr int kCellThreads = 64 + 32 * kEpilogueWarps;
 constexpr int kBarrierBytes = 256;
-constexpr int kBiasBytes = 4 * GRU_POLICY_MAX_HIDDEN * 4;   // four bias vectors, binary32
-constexpr int kCellSmem = kStages * kStageBytes + kBarrierBytes + kBiasBytes + 1024;  // + slack to align
+// dynamic shared memory: the stage ring, the barriers, four binary32 bias vectors, the head's weights
+// as [H][4], slack to align to 1024
+constexpr int cell_smem_bytes(int H, bool with_head)
+{
+    return kStages * kStageBytes + kBarrierBytes + (with_head ? 8 : 4) * H * 4 + 1024;
+}
+constexpr int kMaxSmem = 227 * 1024;   // per block on sm_100
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait
 constexpr unsigned long long kDrainNs = 200000ull;          // let copies in flight land after an abort
 
@@ -95,11 +100,6 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
                  : "memory");
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
@@ -301,6 +301,8 @@ struct CellArgs {
     const float *b_z;   // -log2(e) * (b_iz + b_hz)
     const float *b_in;
     const float *b_hn;
+    const float *head_w4;   // [H][4]: the head's weights by hidden unit, or nullptr (no partial sums)
+    float4 *partial;        // [n][H/32]: the head's partial sums of each block of 32 units of h'
     int n;
     int H;
     int *err;
@@ -323,6 +325,7 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars_ptr + 16 * kStages + 32);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars_ptr + 16 * kStages + 40);
     float *bias_s = reinterpret_cast<float *>(bars_ptr + kBarrierBytes);   // [4][H]: r, z, in, hn
+    float4 *head_s = reinterpret_cast<float4 *>(bias_s + 4 * a.H);         // [H]: the head's weights of a unit
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_cta_rank();        // 0 = leader of the pair
@@ -351,6 +354,7 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
         bias_s[a.H + i] = a.b_z[i];
         bias_s[2 * a.H + i] = a.b_in[i];
         bias_s[3 * a.H + i] = a.b_hn[i];
+        if (a.head_w4 != nullptr) head_s[i] = reinterpret_cast<const float4 *>(a.head_w4)[i];
     }
     tc_fence_before_sync();
     cluster_sync_all();          // both blocks' barriers and tensor memory exist from here on
@@ -461,6 +465,7 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
             const size_t off = static_cast<size_t>(live ? row : 0) * a.H + static_cast<size_t>(j) * kHT;
             const uint4 *hrow = reinterpret_cast<const uint4 *>(a.h_in + off);
             uint4 *orow = reinterpret_cast<uint4 *>(a.h_out + off);
+            float part[3] = {0.0f, 0.0f, 0.0f};   // the head's partial sums over this warp's 32 units
 #pragma unroll 1
             for (int c = c_begin; c < c_begin + kHT / 2; c += 16) {
                 uint32_t nx[16], r[16], z[16], nh[16];
@@ -502,12 +507,27 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
                     }
                     ow[i4 / 2] = pack_bf16(o[0], o[1]);
                     ow[i4 / 2 + 1] = pack_bf16(o[2], o[3]);
+                    if (a.head_w4 != nullptr) {
+                        // the head sees h' as stored: rounded to bfloat16
+                        const float hr[4] = {bf16_lo(ow[i4 / 2]), bf16_hi(ow[i4 / 2]), bf16_lo(ow[i4 / 2 + 1]),
+                                             bf16_hi(ow[i4 / 2 + 1])};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float4 wv = head_s[j * kHT + c + i4 + e];
+                            part[0] = __fmaf_rn(hr[e], wv.x, part[0]);
+                            part[1] = __fmaf_rn(hr[e], wv.y, part[1]);
+                            part[2] = __fmaf_rn(hr[e], wv.z, part[2]);
+                        }
+                    }
                 }
                 if (live) {
                     orow[c / 8] = make_uint4(ow[0], ow[1], ow[2], ow[3]);
                     orow[c / 8 + 1] = make_uint4(ow[4], ow[5], ow[6], ow[7]);
                 }
             }
+            if (a.head_w4 != nullptr && live)
+                a.partial[static_cast<size_t>(row) * (a.H / 32) + (j * kHT + c_begin) / 32] =
+                    make_float4(part[0], part[1], part[2], 0.0f);
             tmem_wait_st();
             tc_fence_before_sync();
             __syncwarp();
@@ -608,12 +628,13 @@ struct EncodeTable<0> {
     static EncodeKernel get(int) { return nullptr; }
 };
 
-// 128 envs per block, one thread per env: logits[a] = fma chain over the hidden units
-// in ascending order.  The block brings 64 units of its 128 rows at a time through
+// 64 envs per block, one thread per env.  logits[a] = bias + the partial sums of the blocks of
+// 32 hidden units in block order, a partial sum being an fma chain from zero over its units in
+// ascending order.  The block brings 64 units of its 64 rows at a time through
 // shared memory with coalesced loads (rows padded to 33 words so that a thread walking
 // its own row meets no bank conflict); the head's weights sit in shared memory as
 // [unit][AP] so that one 16-byte broadcast load feeds up to four chains.
-constexpr int kHeadRows = 128;
+constexpr int kHeadRows = 64;    // small blocks: they fit beside a cell block on an SM
 constexpr int kHeadPitch = 33;   // words per staged row: 32 data + 1 pad
 
 template <int AP>   // actions padded to 4 or 8
@@ -630,9 +651,12 @@ k_head(const __nv_bfloat16 *__restrict__ h, float *__restrict__ logits, const fl
     }
     const int m0 = blockIdx.x * kHeadRows;
     const int m = m0 + threadIdx.x;
-    float acc[AP];
+    float total[AP], acc[AP];
 #pragma unroll
-    for (int a = 0; a < AP; ++a) acc[a] = a < A ? __ldg(head_b + a) : 0.0f;
+    for (int a = 0; a < AP; ++a) {
+        total[a] = a < A ? __ldg(head_b + a) : 0.0f;
+        acc[a] = 0.0f;
+    }
     for (int k0 = 0; k0 < H; k0 += 64) {
         __syncthreads();   // the previous chunk has been read (and, first time, w_s is complete)
 #pragma unroll
@@ -666,13 +690,43 @@ k_head(const __nv_bfloat16 *__restrict__ h, float *__restrict__ logits, const fl
                     acc[4 * a4 + 3] = __fmaf_rn(hv[e], wv.w, acc[4 * a4 + 3]);
                 }
             }
+            if ((p & 15) == 15) {   // a block of 32 units ends
+#pragma unroll
+                for (int a = 0; a < AP; ++a) {
+                    total[a] = __fadd_rn(total[a], acc[a]);
+                    acc[a] = 0.0f;
+                }
+            }
         }
     }
     if (m < n) {
 #pragma unroll
         for (int a = 0; a < AP; ++a)
-            if (a < A) logits[static_cast<size_t>(m) * A + a] = acc[a];
+            if (a < A) logits[static_cast<size_t>(m) * A + a] = total[a];
     }
+}
+
+// logits[a] = bias + the cell kernel's partial sums in block order (A <= 4).
+__global__ void __launch_bounds__(256)
+k_head_reduce(const float4 *__restrict__ partial, float *__restrict__ logits, const float *__restrict__ head_b,
+              int n, int blocks, int A)
+{
+    const int m = blockIdx.x * blockDim.x + threadIdx.x;
+    if (m >= n) return;
+    float total[4];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) total[a] = a < A ? __ldg(head_b + a) : 0.0f;
+    const float4 *row = partial + static_cast<size_t>(m) * blocks;
+    for (int b = 0; b < blocks; ++b) {
+        const float4 v = __ldg(row + b);
+        total[0] = __fadd_rn(total[0], v.x);
+        total[1] = __fadd_rn(total[1], v.y);
+        total[2] = __fadd_rn(total[2], v.z);
+        total[3] = __fadd_rn(total[3], v.w);
+    }
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+        if (a < A) logits[static_cast<size_t>(m) * A + a] = total[a];
 }
 
 // ---------------------------------------------------------------- host side
@@ -731,6 +785,7 @@ struct gru_policy {
     __nv_bfloat16 *wx = nullptr, *wh = nullptr;   // packed [H/64][192][H]
     float *b_r = nullptr, *b_z = nullptr, *b_in = nullptr, *b_hn = nullptr;
     float *enc_w = nullptr, *enc_b = nullptr, *head_w = nullptr, *head_b = nullptr;
+    float *head_w4 = nullptr;   // [H][4], for the cell kernel's partial sums (n_actions <= 4)
     int *err = nullptr;
     CUtensorMap tm_wx, tm_wh;
 };
@@ -756,6 +811,7 @@ void release(gru_policy *p)
     cudaFree(p->enc_b);
     cudaFree(p->head_w);
     cudaFree(p->head_b);
+    cudaFree(p->head_w4);
     cudaFree(p->err);
     delete p;
 }
@@ -818,19 +874,24 @@ int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions, 
         b_in[c] = b_ih[2 * H + c];
         b_hn[c] = b_hh[2 * H + c];
     }
+    std::vector<float> head_w4(static_cast<size_t>(H) * 4, 0.0f);
+    for (int c = 0; c < H; ++c)
+        for (int act = 0; act < n_actions && act < 4; ++act) head_w4[static_cast<size_t>(c) * 4 + act] = head_w[static_cast<size_t>(act) * H + c];
     bool ok = upload(&p->wx, wx) && upload(&p->wh, wh) && upload(&p->b_r, b_r) && upload(&p->b_z, b_z) &&
               upload(&p->b_in, b_in) && upload(&p->b_hn, b_hn) &&
               upload(&p->enc_w, std::vector<float>(enc_w, enc_w + static_cast<size_t>(H) * obs_dim)) &&
               upload(&p->enc_b, std::vector<float>(enc_b, enc_b + H)) &&
               upload(&p->head_w, std::vector<float>(head_w, head_w + static_cast<size_t>(n_actions) * H)) &&
               upload(&p->head_b, std::vector<float>(head_b, head_b + n_actions)) &&
+              upload(&p->head_w4, head_w4) &&
               upload(&p->err, std::vector<int>(1, 0));
     if (ok) {
         TensorMapEncodeFn enc = tensor_map_encoder();
         ok = encode_operand(enc, &p->tm_wx, p->wx, H, static_cast<uint64_t>(3) * H, kBRows) &&
              encode_operand(enc, &p->tm_wh, p->wh, H, static_cast<uint64_t>(3) * H, kBRows);
     }
-    if (ok) ok = cudaFuncSetAttribute(k_gru_cell, cudaFuncAttributeMaxDynamicSharedMemorySize, kCellSmem) ==
+    if (ok) ok = cudaFuncSetAttribute(k_gru_cell, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      cell_smem_bytes(H, cell_smem_bytes(H, true) <= kMaxSmem)) ==
                  cudaSuccess;
     // Ask for the largest shared-memory partition, not the smallest that holds one block, so that
     // small blocks of other kernels can share an SM with a cell block.
@@ -841,7 +902,7 @@ int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions, 
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(static_cast<unsigned>(p->sms & ~1));
         cfg.blockDim = dim3(kCellThreads);
-        cfg.dynamicSmemBytes = kCellSmem;
+        cfg.dynamicSmemBytes = cell_smem_bytes(H, cell_smem_bytes(H, true) <= kMaxSmem);
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
@@ -899,12 +960,12 @@ int gru_policy_encode(gru_policy *p, const float *obs, const uint8_t *done, void
     return GRU_POLICY_OK;
 }
 
-int gru_policy_cell(gru_policy *p, const void *x, const void *h_in, void *h_out, int n)
+static int launch_cell(gru_policy *p, const void *x, const void *h_in, void *h_out, float4 *partial, int n)
 {
     if (p == nullptr || x == nullptr || h_in == nullptr || h_out == nullptr) return GRU_POLICY_ENULL;
     if (n < 1) return GRU_POLICY_EINVAL;
     if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(h_in) |
-         reinterpret_cast<uintptr_t>(h_out)) % 16 != 0)
+         reinterpret_cast<uintptr_t>(h_out) | reinterpret_cast<uintptr_t>(partial)) % 16 != 0)
         return GRU_POLICY_EALIGN;
     if (h_out == x || h_out == h_in) return GRU_POLICY_EINVAL;
     TensorMapEncodeFn enc = tensor_map_encoder();
@@ -918,6 +979,8 @@ int gru_policy_cell(gru_policy *p, const void *x, const void *h_in, void *h_out,
     a.b_z = p->b_z;
     a.b_in = p->b_in;
     a.b_hn = p->b_hn;
+    a.head_w4 = partial != nullptr ? p->head_w4 : nullptr;
+    a.partial = partial;
     a.n = n;
     a.H = p->H;
     a.err = p->err;
@@ -926,7 +989,7 @@ int gru_policy_cell(gru_policy *p, const void *x, const void *h_in, void *h_out,
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(static_cast<unsigned>(2 * pairs));
     cfg.blockDim = dim3(kCellThreads);
-    cfg.dynamicSmemBytes = kCellSmem;
+    cfg.dynamicSmemBytes = cell_smem_bytes(p->H, partial != nullptr);
     cfg.stream = p->stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -943,6 +1006,31 @@ int gru_policy_cell(gru_policy *p, const void *x, const void *h_in, void *h_out,
         cudaGetLastError();
         return GRU_POLICY_ECUDA;
     }
+    p->launches += 1;
+    return GRU_POLICY_OK;
+}
+
+int gru_policy_cell(gru_policy *p, const void *x, const void *h_in, void *h_out, int n)
+{
+    return launch_cell(p, x, h_in, h_out, nullptr, n);
+}
+
+size_t gru_policy_workspace_bytes(const gru_policy *p, int n)
+{
+    if (p == nullptr || n < 1) return 0;
+    return static_cast<size_t>(n) * (p->H / 32) * sizeof(float4);
+}
+
+int gru_policy_cell_head(gru_policy *p, const void *x, const void *h_in, void *h_out, float *logits,
+                         void *workspace, int n)
+{
+    if (p == nullptr || logits == nullptr || workspace == nullptr) return GRU_POLICY_ENULL;
+    if (p->A > 4 || cell_smem_bytes(p->H, true) > kMaxSmem) return GRU_POLICY_EINVAL;
+    const int rc = launch_cell(p, x, h_in, h_out, static_cast<float4 *>(workspace), n);
+    if (rc != GRU_POLICY_OK) return rc;
+    k_head_reduce<<<(n + 255) / 256, 256, 0, p->stream>>>(static_cast<const float4 *>(workspace), logits,
+                                                          p->head_b, n, p->H / 32, p->A);
+    if (cudaGetLastError() != cudaSuccess) return GRU_POLICY_ECUDA;
     p->launches += 1;
     return GRU_POLICY_OK;
 }

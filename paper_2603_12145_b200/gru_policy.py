@@ -13,8 +13,8 @@ import numpy as np
 from . import build as _build
 
 EXPORTS = ("gru_policy_create", "gru_policy_destroy", "gru_policy_set_stream", "gru_policy_encode",
-           "gru_policy_cell", "gru_policy_head", "gru_policy_status", "gru_policy_hidden",
-           "gru_policy_launch_count", "gru_policy_strerror")
+           "gru_policy_cell", "gru_policy_head", "gru_policy_workspace_bytes", "gru_policy_cell_head",
+           "gru_policy_status", "gru_policy_hidden", "gru_policy_launch_count", "gru_policy_strerror")
 
 PARAMETERS = ("enc_w", "enc_b", "w_ih", "w_hh", "b_ih", "b_hh", "head_w", "head_b")
 
@@ -47,6 +47,9 @@ def load(build_if_missing: bool = False):
     L.gru_policy_encode.argtypes = [vp, vp, vp, vp, vp, i32]
     L.gru_policy_cell.argtypes = [vp, vp, vp, vp, i32]
     L.gru_policy_head.argtypes = [vp, vp, vp, i32]
+    L.gru_policy_workspace_bytes.argtypes = [vp, i32]
+    L.gru_policy_workspace_bytes.restype = ctypes.c_size_t
+    L.gru_policy_cell_head.argtypes = [vp, vp, vp, vp, vp, vp, i32]
     L.gru_policy_status.argtypes = [vp]
     L.gru_policy_hidden.argtypes = [vp]
     L.gru_policy_launch_count.argtypes = [vp]
@@ -54,7 +57,7 @@ def load(build_if_missing: bool = False):
     L.gru_policy_strerror.argtypes = [i32]
     L.gru_policy_strerror.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("gru_policy_launch_count", "gru_policy_strerror"):
+        if name not in ("gru_policy_launch_count", "gru_policy_strerror", "gru_policy_workspace_bytes"):
             getattr(L, name).restype = i32
     _lib = L
     return L
@@ -109,6 +112,15 @@ def gru_policy_cell(h: int, x, h_in, h_out, n: int) -> None:
 
 def gru_policy_head(h: int, hidden_state, logits, n: int) -> None:
     _check(load().gru_policy_head(h, _ptr(hidden_state), _ptr(logits), int(n)), "gru_policy_head")
+
+
+def gru_policy_workspace_bytes(h: int, n: int) -> int:
+    return int(load().gru_policy_workspace_bytes(h, int(n)))
+
+
+def gru_policy_cell_head(h: int, x, h_in, h_out, logits, workspace, n: int) -> None:
+    _check(load().gru_policy_cell_head(h, _ptr(x), _ptr(h_in), _ptr(h_out), _ptr(logits), _ptr(workspace),
+                                       int(n)), "gru_policy_cell_head")
 
 
 def gru_policy_status(h: int) -> None:
@@ -175,6 +187,25 @@ class GruPolicy:
         self._stream()
         gru_policy_cell(self.h, x, h_in, h_out, n)
         return h_out
+
+    def workspace(self, n: int):
+        """Device scratch for cell_head at n envs."""
+        t = self.torch
+        return t.empty((gru_policy_workspace_bytes(self.h, n),), dtype=t.uint8, device=self.device)
+
+    def cell_head(self, x, h_in, h_out=None, logits=None, workspace=None):
+        """(h_out, logits): the cell and the head of its result in one pass."""
+        t = self.torch
+        n = x.shape[0]
+        if h_out is None:
+            h_out = t.empty((n, self.hidden), dtype=t.bfloat16, device=self.device)
+        if logits is None:
+            logits = t.empty((n, self.n_actions), dtype=t.float32, device=self.device)
+        if workspace is None:
+            workspace = self.workspace(n)
+        self._stream()
+        gru_policy_cell_head(self.h, x, h_in, h_out, logits, workspace, n)
+        return h_out, logits
 
     def head(self, hidden_state, logits=None):
         t = self.torch

@@ -7,10 +7,10 @@ This is the setting of the paper's "GRU rollout (~2M-parameter policy)" rows
 environment the step time is dominated by the model (Sec. 4, time breakdown).
 Per agent step, five kernels of this package and nothing else:
 
-    x       <- gru_policy_encode(obs, done, h)      also clears h where the last step ended an episode
-    h'      <- gru_policy_cell(x, h)                tensor cores
-    logits  <- gru_policy_head(h')
-    actions <- pong_sample_actions(logits, words[i])
+    x          <- gru_policy_encode(obs, done, h)      also clears h where the last step ended an episode
+    h', logits <- gru_policy_cell_head(x, h)           tensor cores; the head's partial sums are formed in
+                                                       the cell's epilogue, a small kernel adds them up
+    actions    <- pong_sample_actions(logits, words[i])
     obs, reward, done <- pong_step(actions)
 
 The uniform numbers of the draws are generated before each replay with
@@ -43,6 +43,7 @@ class PolicyLoop:
         self.h = [torch.zeros((n, H), dtype=torch.bfloat16, device=dev) for _ in range(2)]
         self.cur = 0                                     # which of the two holds the current hidden state
         self.logits = torch.zeros((n, 3), dtype=torch.float32, device=dev)
+        self.scratch = policy.workspace(n)                # the head's partial sums, written by the cell kernel
         self.actions = torch.empty((n,), dtype=torch.uint8, device=dev)
         self.words = torch.empty((self.K, n), dtype=torch.int32, device=dev)
         self.graph = None
@@ -59,9 +60,9 @@ class PolicyLoop:
         if with_policy:
             p = self.policy.h
             gru_policy.gru_policy_encode(p, self.obs, self.done, self.h[self.cur], self.x, n)
-            gru_policy.gru_policy_cell(p, self.x, self.h[self.cur], self.h[self.cur ^ 1], n)
+            gru_policy.gru_policy_cell_head(p, self.x, self.h[self.cur], self.h[self.cur ^ 1], self.logits,
+                                            self.scratch, n)
             self.cur ^= 1
-            gru_policy.gru_policy_head(p, self.h[self.cur], self.logits, n)
         if with_env:
             pong.pong_sample_actions(self.env.h, self.logits, self.words[i], self.actions)
             pong.pong_step(self.env.h, self.actions, self.obs, self.reward, self.done)

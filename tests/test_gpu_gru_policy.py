@@ -162,6 +162,25 @@ def test_head_bit_exact(torch_cuda, H, n):
     pol.close()
 
 
+@pytest.mark.parametrize("H,n", [(64, 1), (576, 700), (128, 513)])
+def test_cell_head_equals_cell_then_head(torch_cuda, H, n):
+    """The fused entry point gives the bits of the two separate calls (whose parity with
+    the oracle the tests above establish)."""
+    torch = torch_cuda
+    w = policy_weights(H, 61)
+    x, h = policy_activations(n, H, 62)
+    pol = gp.GruPolicy(w)
+    xd, hd = to_dev_bf16(torch, x), to_dev_bf16(torch, h)
+    h1 = pol.cell(xd, hd)
+    l1 = pol.head(h1)
+    h2, l2 = pol.cell_head(xd, hd)
+    pol.status()
+    assert torch.equal(h1, h2)
+    assert torch.equal(l1, l2)
+    assert gp.gru_policy_workspace_bytes(pol.h, n) == n * (H // 32) * 16
+    pol.close()
+
+
 def test_argument_errors(torch_cuda):
     torch = torch_cuda
     w = policy_weights(64, 51)

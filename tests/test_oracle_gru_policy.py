@@ -176,6 +176,22 @@ def test_head_against_float64_and_exact_small_integers():
     assert np.array_equal(out[:, 1], h[:, 7]) and not out[:, 0].any() and not out[:, 2].any()
 
 
+def test_head_block_structure_by_a_case_where_the_order_shows():
+    # unit 0 contributes 2^24; units 32..63 (the second block of 32) contribute 1 each.  Added
+    # one by one to 2^24 every 1 would be rounded away (ties to even); as a block they arrive
+    # as 32, which 2^24 can absorb exactly.
+    H = 64
+    h = np.zeros((1, H), np.float32); w = np.zeros((3, H), np.float32)
+    h[0, 0] = 4096.0; w[0, 0] = 4096.0
+    h[0, 32:] = 1.0; w[0, 32:] = 1.0
+    w[1, 0] = 4096.0; w[1, 1:33] = 1.0; h[0, 1:32] = 0.0      # row 1: the ones sit across both blocks
+    out = gp.head(h, w, np.array([0.0, 0.0, 0.5], np.float32))
+    assert out[0, 0] == 2.0 ** 24 + 32.0
+    # row 1: block 0 holds 2^24 (unit 0) and nothing else that is non-zero in h; block 1 holds unit 32 only
+    assert out[0, 1] == 2.0 ** 24                       # 2^24 + 1 is a tie: to even
+    assert out[0, 2] == 0.5
+
+
 def test_generated_parameters_are_bfloat16_representable():
     w = policy_weights(128, 14)
     x, h = policy_activations(7, 128, 15)
