@@ -561,6 +561,50 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
 constexpr int kEncodeRows = 4;
 constexpr int kEncodeCols = 4;
 
+// One pass of a thread: `rows` consecutive envs starting at m0 (FULL: exactly kEncodeRows, so
+// that every offset is a compile-time constant).
+template <int OD, bool FULL>
+__device__ __forceinline__ void encode_pass(const float *__restrict__ row, const uint8_t *__restrict__ done_m0,
+                                            __nv_bfloat16 *__restrict__ hrow, __nv_bfloat16 *__restrict__ xrow,
+                                            const float (&w)[kEncodeCols][OD], const float (&b)[kEncodeCols],
+                                            int rows, int H)
+{
+    float o[kEncodeRows][OD];
+    bool ended[kEncodeRows];
+    // all loads of the pass first; a short last pass re-reads its first env
+#pragma unroll
+    for (int r = 0; r < kEncodeRows; ++r) {
+        const int rr = FULL ? r : (r < rows ? r : 0);
+        if constexpr (OD % 2 == 0) {   // rows are 8-byte aligned: load pairs
+#pragma unroll
+            for (int i = 0; i < OD; i += 2) {
+                const float2 v = __ldg(reinterpret_cast<const float2 *>(row + rr * OD + i));
+                o[r][i] = v.x;
+                o[r][i + 1] = v.y;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < OD; ++i) o[r][i] = __ldg(row + rr * OD + i);
+        }
+        ended[r] = done_m0 != nullptr && __ldg(done_m0 + rr) != 0;
+    }
+#pragma unroll
+    for (int r = 0; r < kEncodeRows; ++r) {
+        if (!FULL && r >= rows) break;
+        float v[kEncodeCols];
+#pragma unroll
+        for (int e = 0; e < kEncodeCols; ++e) {
+            float acc = b[e];
+#pragma unroll
+            for (int i = 0; i < OD; ++i) acc = __fmaf_rn(o[r][i], w[e][i], acc);
+            v[e] = fmaxf(acc, 0.0f);
+        }
+        *reinterpret_cast<uint2 *>(xrow + static_cast<size_t>(r) * H) =
+            make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
+        if (ended[r]) *reinterpret_cast<uint2 *>(hrow + static_cast<size_t>(r) * H) = make_uint2(0u, 0u);
+    }
+}
+
 template <int OD>
 __global__ void __launch_bounds__(GRU_POLICY_MAX_HIDDEN / kEncodeCols)
 k_encode(const float *__restrict__ obs, const uint8_t *__restrict__ done, __nv_bfloat16 *__restrict__ h,
@@ -579,40 +623,14 @@ k_encode(const float *__restrict__ obs, const uint8_t *__restrict__ done, __nv_b
     const bool mask = done != nullptr && h != nullptr;
     for (long long m0 = static_cast<long long>(blockIdx.x) * kEncodeRows; m0 < n;
          m0 += static_cast<long long>(gridDim.x) * kEncodeRows) {
-        float o[kEncodeRows][OD];
-        bool ended[kEncodeRows];
-#pragma unroll
-        for (int r = 0; r < kEncodeRows; ++r) {
-            const long long m = m0 + r < n ? m0 + r : n - 1;
-            const float *row = obs + static_cast<size_t>(m) * OD;
-            if constexpr (OD % 2 == 0) {   // rows are 8-byte aligned: load pairs
-#pragma unroll
-                for (int i = 0; i < OD; i += 2) {
-                    const float2 v = __ldg(reinterpret_cast<const float2 *>(row + i));
-                    o[r][i] = v.x;
-                    o[r][i + 1] = v.y;
-                }
-            } else {
-#pragma unroll
-                for (int i = 0; i < OD; ++i) o[r][i] = __ldg(row + i);
-            }
-            ended[r] = mask && __ldg(done + m) != 0;
-        }
-#pragma unroll
-        for (int r = 0; r < kEncodeRows; ++r) {
-            if (m0 + r >= n) break;
-            float v[kEncodeCols];
-#pragma unroll
-            for (int e = 0; e < kEncodeCols; ++e) {
-                float acc = b[e];
-#pragma unroll
-                for (int i = 0; i < OD; ++i) acc = __fmaf_rn(o[r][i], w[e][i], acc);
-                v[e] = acc > 0.0f ? acc : 0.0f;
-            }
-            const size_t off = static_cast<size_t>(m0 + r) * H + c;
-            *reinterpret_cast<uint2 *>(x_out + off) = make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
-            if (ended[r]) *reinterpret_cast<uint2 *>(h + off) = make_uint2(0u, 0u);
-        }
+        const float *row = obs + static_cast<size_t>(m0) * OD;
+        const uint8_t *done_m0 = mask ? done + m0 : nullptr;
+        __nv_bfloat16 *xrow = x_out + static_cast<size_t>(m0) * H + c;
+        __nv_bfloat16 *hrow = h + static_cast<size_t>(m0) * H + c;
+        if (n - m0 >= kEncodeRows)
+            encode_pass<OD, true>(row, done_m0, hrow, xrow, w, b, kEncodeRows, H);
+        else
+            encode_pass<OD, false>(row, done_m0, hrow, xrow, w, b, static_cast<int>(n - m0), H);
     }
 }
 
@@ -780,6 +798,7 @@ struct gru_policy {
     int device = 0, sms = 0;
     int pairs = 0;   // clusters of two blocks that can be resident at once
     int top_priority = 0;   // numerically lowest = most urgent launch priority of the device
+    int encode_blocks_per_sm = 0;   // resident encoder blocks per SM, found at the first call
     cudaStream_t stream = nullptr;
     int64_t launches = 0;
     __nv_bfloat16 *wx = nullptr, *wh = nullptr;   // packed [H/64][192][H]
@@ -948,11 +967,21 @@ int gru_policy_encode(gru_policy *p, const float *obs, const uint8_t *done, void
     if (n < 1) return GRU_POLICY_EINVAL;
     if ((reinterpret_cast<uintptr_t>(x_out) | reinterpret_cast<uintptr_t>(h)) % 16 != 0) return GRU_POLICY_EALIGN;
     if (reinterpret_cast<uintptr_t>(obs) % 8 != 0) return GRU_POLICY_EALIGN;
-    const long long passes = (static_cast<long long>(n) + kEncodeRows - 1) / kEncodeRows;
-    const long long cap = static_cast<long long>(p->sms) * 8;
-    const unsigned blocks = static_cast<unsigned>(passes < cap ? passes : cap);
     const unsigned threads = static_cast<unsigned>((p->H / kEncodeCols + 31) / 32 * 32);
-    EncodeTable<GRU_POLICY_MAX_OBS>::get(p->obs_dim)<<<blocks, threads, 0, p->stream>>>(
+    EncodeKernel kernel = EncodeTable<GRU_POLICY_MAX_OBS>::get(p->obs_dim);
+    if (p->encode_blocks_per_sm == 0) {   // one full wave of resident blocks: no partial second wave
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, static_cast<int>(threads), 0) != cudaSuccess ||
+            per_sm < 1) {
+            cudaGetLastError();
+            per_sm = 4;
+        }
+        p->encode_blocks_per_sm = per_sm;
+    }
+    const long long passes = (static_cast<long long>(n) + kEncodeRows - 1) / kEncodeRows;
+    const long long cap = static_cast<long long>(p->sms) * p->encode_blocks_per_sm;
+    const unsigned blocks = static_cast<unsigned>(passes < cap ? passes : cap);
+    kernel<<<blocks, threads, 0, p->stream>>>(
         obs, done, static_cast<__nv_bfloat16 *>(h), static_cast<__nv_bfloat16 *>(x_out), p->enc_w, p->enc_b, n,
         p->H);
     if (cudaGetLastError() != cudaSuccess) return GRU_POLICY_ECUDA;
