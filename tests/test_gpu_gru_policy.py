@@ -181,6 +181,44 @@ def test_cell_head_equals_cell_then_head(torch_cuda, H, n):
     pol.close()
 
 
+def test_other_shapes_odd_obs_dim_and_eight_actions(torch_cuda):
+    """obs_dim 5 takes the scalar-load path of the encoder, 8 actions the two-vector path of the head;
+    hidden 896 is the largest the fused entry point takes, 960 must be refused by it."""
+    torch = torch_cuda
+    H, n = 192, 777
+    w = policy_weights(H, 71, obs_dim=5, n_actions=8)
+    rng = np.random.Generator(np.random.PCG64(72))
+    obs = rng.uniform(-1.0, 1.0, (n, 5)).astype(np.float32)
+    hvals = bf16_values((n, H), 73, -7, 0)
+    pol = gp.GruPolicy(w)
+    x = pol.encode(torch.from_numpy(obs).cuda())
+    assert np.array_equal(from_dev_bf16(torch, x).view(np.uint32),
+                          ogp.encode(obs, w["enc_w"], w["enc_b"]).view(np.uint32))
+    logits = pol.head(to_dev_bf16(torch, hvals))
+    assert np.array_equal(logits.cpu().numpy().view(np.uint32),
+                          ogp.head(hvals, w["head_w"], w["head_b"]).view(np.uint32))
+    with pytest.raises(gp.GruPolicyError) as e:      # more than 4 actions: not through the fused call
+        pol.cell_head(x, to_dev_bf16(torch, hvals))
+    assert e.value.code == -1
+    pol.status(); pol.close()
+    for H, fused in ((896, True), (960, False)):
+        w = policy_weights(H, 74)
+        xs, hs = policy_activations(130, H, 75)
+        pol = gp.GruPolicy(w)
+        xd, hd = to_dev_bf16(torch, xs), to_dev_bf16(torch, hs)
+        h1 = pol.cell(xd, hd)
+        want = ogp.cell(xs, hs, w["w_ih"], w["w_hh"], w["b_ih"], w["b_hh"])
+        assert np.all(np.abs(from_dev_bf16(torch, h1) - want) <= cell_tolerance(want))
+        if fused:
+            h2, l2 = pol.cell_head(xd, hd)
+            assert torch.equal(h1, h2) and torch.equal(l2, pol.head(h1))
+        else:
+            with pytest.raises(gp.GruPolicyError) as e:
+                pol.cell_head(xd, hd)
+            assert e.value.code == -1
+        pol.status(); pol.close()
+
+
 def test_argument_errors(torch_cuda):
     torch = torch_cuda
     w = policy_weights(64, 51)
@@ -203,5 +241,17 @@ def test_argument_errors(torch_cuda):
     with pytest.raises(gp.GruPolicyError) as e:
         gp.gru_policy_cell(pol.h, x, h, out, 0)
     assert e.value.code == -1
+    logits = torch.zeros((8, 3), device="cuda")
+    ws = pol.workspace(8)
+    with pytest.raises(gp.GruPolicyError) as e:      # scratch must be 16-byte aligned
+        gp.gru_policy_cell_head(pol.h, x, h, out, logits, ws.data_ptr() + 4, 8)
+    assert e.value.code == -3
+    with pytest.raises(gp.GruPolicyError) as e:
+        gp.gru_policy_cell_head(pol.h, x, h, out, logits, None, 8)
+    assert e.value.code == -2
+    obs = torch.zeros((9, 6), device="cuda")
+    with pytest.raises(gp.GruPolicyError) as e:      # obs rows are read in pairs: 8-byte alignment
+        gp.gru_policy_encode(pol.h, obs.data_ptr() + 4, None, None, x, 8)
+    assert e.value.code == -3
     pol.status()
     pol.close()
