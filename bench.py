@@ -168,6 +168,9 @@ def oracle_sample(w):
     import oracle
     from paper_2603_12145_b200.inputs import explicit_actions
     n_sample = min(w["n"], 256 if w["obs_mode"] == 1 else 8192)
+    if w.get("env") == "policy":
+        n_sample = 64
+        return None, n_sample, policy_oracle_call(n_sample, w["T"])
     if w.get("env") == "cartpole":
         from oracle import cartpole as oracle_cartpole
         o = oracle_cartpole.OracleCartPole(n_sample, SEED)
@@ -177,6 +180,31 @@ def oracle_sample(w):
         acts = explicit_actions(w["T"], n_sample, seed=SEED)
         return o, n_sample, (lambda: o.rollout(w["T"], 2, acts))
     return o, n_sample, (lambda: o.rollout(w["T"], w["mode"]))
+
+
+def policy_oracle_call(n_sample, T, hidden=576):
+    """The whole agent step from the oracles alone (encoder, binary64 cell rounded once to
+    bfloat16, head, sampling, env step), T steps per call on the first n_sample envs."""
+    import numpy as np
+    import oracle
+    from oracle import gru_policy as ogp
+    from paper_2603_12145_b200.inputs import policy_weights
+    p = policy_weights(hidden, SEED)
+    o = oracle.OraclePong(n_sample, SEED)
+    state = {"obs": o.reset(), "h": np.zeros((n_sample, hidden), np.float32)}
+
+    def call():
+        words = o.fill_words(T)
+        obs, h = state["obs"], state["h"]
+        for i in range(T):
+            x = ogp.encode(obs, p["enc_w"], p["enc_b"])
+            h = ogp.bf16_round_f64(ogp.cell(x, h, p["w_ih"], p["w_hh"], p["b_ih"], p["b_hh"]))
+            logits = ogp.head(h, p["head_w"], p["head_b"])
+            obs, _, done = o.step(oracle.sample_actions(logits, words[i]))
+            h[done != 0] = 0.0
+        state["obs"], state["h"] = obs, h
+
+    return call
 
 
 def cpu_oracle_rate(w, budget_s):
@@ -220,7 +248,8 @@ def run_reference(args, rank):
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": done_steps, "warmup": max(args.warmup, 1), "ms_per_step": dt / done_steps * 1e3,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": {"policy": "f64 cell, f32 encoder and head, int32 env", "cartpole": "f32"}.get(w.get("env"), "int32"),
         "data": "synthetic", "config": {"workload": WORKLOAD, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -234,8 +263,6 @@ def run_policy(args, w, rank, world, local):
     import torch
     from paper_2603_12145_b200 import gru_policy, policy_loop, pong, sharding
     from paper_2603_12145_b200.inputs import policy_weights
-    import oracle
-    from oracle import gru_policy as ogp
     import numpy as np
 
     N, K = w["n"], w["T"]
@@ -310,18 +337,11 @@ def run_policy(args, w, rank, world, local):
     if rank != 0:
         return
     # CPU: the whole agent step from the oracles (encoder, binary64 cell, head, sampling, env step)
-    n_s = 256
-    o = oracle.OraclePong(n_s, SEED)
-    obs = o.reset()
-    h = np.zeros((n_s, hidden), np.float32)
+    n_s = 64
+    call = policy_oracle_call(n_s, 1, hidden)
     c0, reps = time.perf_counter(), 0
     while time.perf_counter() - c0 < max(args.cpu_seconds, 0.2):
-        words = o.fill_words(1)
-        x = ogp.encode(obs, params["enc_w"], params["enc_b"])
-        h = ogp.bf16_round_f64(ogp.cell(x, h, params["w_ih"], params["w_hh"], params["b_ih"], params["b_hh"]))
-        logits = ogp.head(h, params["head_w"], params["head_b"])
-        obs, _, done = o.step(oracle.sample_actions(logits, words[0]))
-        h[done != 0] = 0.0
+        call()
         reps += 1
     cpu_dt = time.perf_counter() - c0
     line = {
