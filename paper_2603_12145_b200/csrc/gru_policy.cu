@@ -650,7 +650,8 @@ struct EncodeTable<0> {
 // 32 hidden units in block order, a partial sum being an fma chain from zero over its units in
 // ascending order.  The block brings 64 units of its 64 rows at a time through
 // shared memory with coalesced loads (rows padded to 33 words so that a thread walking
-// its own row meets no bank conflict); the head's weights sit in shared memory as
+// its own row meets no bank conflict), the next chunk's loads in flight while the
+// current one is summed; the head's weights sit in shared memory as
 // [unit][AP] so that one 16-byte broadcast load feeds up to four chains.
 constexpr int kHeadRows = 64;    // small blocks: they fit beside a cell block on an SM
 constexpr int kHeadPitch = 33;   // words per staged row: 32 data + 1 pad
@@ -675,22 +676,32 @@ k_head(const __nv_bfloat16 *__restrict__ h, float *__restrict__ logits, const fl
         total[a] = a < A ? __ldg(head_b + a) : 0.0f;
         acc[a] = 0.0f;
     }
+    // this thread's eight 16-byte pieces of a 64-unit chunk of the block's rows
+    auto fetch = [&](int k0, uint4 (&v)[8]) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int piece = i * kHeadRows + threadIdx.x;   // 8 pieces per row
+            const int row = piece >> 3, seg = piece & 7;
+            v[i] = make_uint4(0, 0, 0, 0);
+            if (m0 + row < n)
+                v[i] = __ldg(reinterpret_cast<const uint4 *>(h + static_cast<size_t>(m0 + row) * H + k0) + seg);
+        }
+    };
+    uint4 next[8];
+    fetch(0, next);
     for (int k0 = 0; k0 < H; k0 += 64) {
         __syncthreads();   // the previous chunk has been read (and, first time, w_s is complete)
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
-            const int piece = i * kHeadRows + threadIdx.x;   // 16-byte pieces, 8 per row
-            const int row = piece >> 3, seg = piece & 7;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (m0 + row < n)
-                v = __ldg(reinterpret_cast<const uint4 *>(h + static_cast<size_t>(m0 + row) * H + k0) + seg);
-            uint32_t *dst = tile + row * kHeadPitch + seg * 4;
-            dst[0] = v.x;
-            dst[1] = v.y;
-            dst[2] = v.z;
-            dst[3] = v.w;
+            const int piece = i * kHeadRows + threadIdx.x;
+            uint32_t *dst = tile + (piece >> 3) * kHeadPitch + (piece & 7) * 4;
+            dst[0] = next[i].x;
+            dst[1] = next[i].y;
+            dst[2] = next[i].z;
+            dst[3] = next[i].w;
         }
         __syncthreads();
+        if (k0 + 64 < H) fetch(k0 + 64, next);   // in flight while this chunk is summed
         const uint32_t *mine = tile + threadIdx.x * kHeadPitch;
         const float4 *wk = reinterpret_cast<const float4 *>(w_s + static_cast<size_t>(k0) * AP);
 #pragma unroll 8
