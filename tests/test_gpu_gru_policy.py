@@ -181,6 +181,27 @@ def test_cell_head_equals_cell_then_head(torch_cuda, H, n):
     pol.close()
 
 
+def test_cell_rows_do_not_depend_on_the_batch(torch_cuda):
+    """A row's result is the same bits whatever the batch it is launched in: task counts below,
+    at and above the number of resident block pairs, ragged last tiles, both entry points."""
+    torch = torch_cuda
+    H, nmax = 576, 20000
+    pol = gp.GruPolicy(policy_weights(H, 81))
+    x, h = policy_activations(nmax, H, 82)
+    xd, hd = to_dev_bf16(torch, x), to_dev_bf16(torch, h)
+    ref_h = torch.empty_like(hd)
+    ref_l = torch.empty((nmax, 3), device="cuda")
+    for a in range(0, nmax, 1024):
+        b = min(nmax, a + 1024)
+        ref_h[a:b], ref_l[a:b] = pol.cell_head(xd[a:b], hd[a:b])
+    for n in (1, 127, 129, 256, 257, 2047, 2105, 2106, 4211, 9472, 18944, 18945, nmax):
+        out, logits = pol.cell_head(xd[:n], hd[:n])
+        assert torch.equal(out, ref_h[:n]) and torch.equal(logits, ref_l[:n]), n
+        assert torch.equal(pol.cell(xd[:n], hd[:n]), ref_h[:n]), n
+    pol.status()
+    pol.close()
+
+
 def test_other_shapes_odd_obs_dim_and_eight_actions(torch_cuda):
     """obs_dim 5 takes the scalar-load path of the encoder, 8 actions the two-vector path of the head;
     hidden 896 is the largest the fused entry point takes, 960 must be refused by it."""
