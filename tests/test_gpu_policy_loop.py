@@ -145,9 +145,9 @@ def test_loop_against_an_independent_oracle_loop(torch):
         assert np.array_equal(loop.reward.cpu().numpy()[same], r[same])
         assert np.array_equal(loop.done.cpu().numpy()[same], done[same])
     pol.status()
-    assert worst_h <= 2.0 ** -6, worst_h          # a few places of 2^-8 relative at |h| <= 1
+    assert worst_h <= 2.0 ** -7, worst_h          # observed: one place (2^-9 at |h| < 1/2); a few are allowed
     assert worst_margin <= 2e-3, worst_margin
-    assert (~same).mean() <= 0.02, (~same).sum()
+    assert (~same).mean() <= 0.01, (~same).sum()  # observed: none
 
 
 def test_pipelined_loop_equals_the_single_loop(torch):
