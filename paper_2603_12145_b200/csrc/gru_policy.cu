@@ -553,97 +553,197 @@ k_gru_cell(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUt
 
 // ---------------------------------------------------------------- encoder and head
 
-// Thread t of a block owns hidden units 4t..4t+3 with their encoder weights in
-// registers; the block walks over envs, four per pass.  A warp's stores cover 256
-// contiguous bytes of a row of x.  Where the env's episode just ended the same four
-// units of h are cleared.  OD = obs_dim, known at compile time so that the fma chain
-// is exactly OD long.
+// Thread t of a block owns the COLS hidden units of group t % (H/COLS), with their encoder
+// weights in registers, and row slot t / (H/COLS) (H/COLS need not be a multiple of 32: the
+// block is H/COLS times a slot count that is).  The block takes chunks of consecutive envs:
+// it brings the weights (once) and the chunk's rows of obs and done bytes into shared memory
+// with coalesced loads, so the loop over the chunk has no global load in it; a slot then
+// takes kEncodeRows consecutive envs per pass.  Each output is the fma chain from the bias in
+// ascending input order, rounded to bfloat16 in pairs; the relu is taken on the packed pair
+// (max with +0: rounding keeps the sign, and -0 and NaN become +0 exactly as with
+// "acc > 0 ? acc : 0" before the rounding).  A thread's store covers 2 * COLS bytes, a warp's
+// 64 * COLS contiguous bytes of a row of x.  Where the env's episode just ended the same units
+// of h are cleared.  OD = obs_dim, known at compile time so that the chain is exactly OD long.
 constexpr int kEncodeRows = 4;
-constexpr int kEncodeCols = 4;
+constexpr int kEncodeMaxThreads = 288;   // two blocks per SM with up to 112 registers per thread
+constexpr int kEncodeMaxChunk = 256;     // envs per chunk, a multiple of kEncodeRows
 
-// One pass of a thread: `rows` consecutive envs starting at m0 (FULL: exactly kEncodeRows, so
-// that every offset is a compile-time constant).
-template <int OD, bool FULL>
-__device__ __forceinline__ void encode_pass(const float *__restrict__ row, const uint8_t *__restrict__ done_m0,
-                                            __nv_bfloat16 *__restrict__ hrow, __nv_bfloat16 *__restrict__ xrow,
-                                            const float (&w)[kEncodeCols][OD], const float (&b)[kEncodeCols],
-                                            int rows, int H)
+__device__ __forceinline__ uint32_t pack_bf16_relu(float lo, float hi)
 {
-    float o[kEncodeRows][OD];
-    bool ended[kEncodeRows];
-    // all loads of the pass first; a short last pass re-reads its first env
-#pragma unroll
-    for (int r = 0; r < kEncodeRows; ++r) {
-        const int rr = FULL ? r : (r < rows ? r : 0);
-        if constexpr (OD % 2 == 0) {   // rows are 8-byte aligned: load pairs
-#pragma unroll
-            for (int i = 0; i < OD; i += 2) {
-                const float2 v = __ldg(reinterpret_cast<const float2 *>(row + rr * OD + i));
-                o[r][i] = v.x;
-                o[r][i + 1] = v.y;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < OD; ++i) o[r][i] = __ldg(row + rr * OD + i);
-        }
-        ended[r] = done_m0 != nullptr && __ldg(done_m0 + rr) != 0;
-    }
-#pragma unroll
-    for (int r = 0; r < kEncodeRows; ++r) {
-        if (!FULL && r >= rows) break;
-        float v[kEncodeCols];
-#pragma unroll
-        for (int e = 0; e < kEncodeCols; ++e) {
-            float acc = b[e];
-#pragma unroll
-            for (int i = 0; i < OD; ++i) acc = __fmaf_rn(o[r][i], w[e][i], acc);
-            v[e] = fmaxf(acc, 0.0f);
-        }
-        *reinterpret_cast<uint2 *>(xrow + static_cast<size_t>(r) * H) =
-            make_uint2(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]));
-        if (ended[r]) *reinterpret_cast<uint2 *>(hrow + static_cast<size_t>(r) * H) = make_uint2(0u, 0u);
-    }
+    const __nv_bfloat162 v = __hmax2(__floats2bfloat162_rn(lo, hi), __floats2bfloat162_rn(0.0f, 0.0f));
+    return *reinterpret_cast<const uint32_t *>(&v);
+}
+
+// 2 * COLS bytes (COLS = 4 or 8) to a suitably aligned address.
+template <int COLS>
+__device__ __forceinline__ void store_units(__nv_bfloat16 *dst, const uint32_t (&v)[COLS / 2])
+{
+    if constexpr (COLS == 8)
+        *reinterpret_cast<uint4 *>(dst) = make_uint4(v[0], v[1], v[2], v[3]);
+    else
+        *reinterpret_cast<uint2 *>(dst) = make_uint2(v[0], v[1]);
 }
 
 template <int OD>
-__global__ void __launch_bounds__(GRU_POLICY_MAX_HIDDEN / kEncodeCols)
+struct EncodeShape {
+    static constexpr int kCols = OD <= 8 ? 8 : 4;   // hidden units per thread: its weights stay in registers
+};
+
+// Shared memory: weights [H][OD] and biases [H] (float4 aligned), then the chunk's obs
+// [chunk][OD] and its done bytes [chunk].
+template <int OD>
+__global__ void __launch_bounds__(kEncodeMaxThreads, 2)
 k_encode(const float *__restrict__ obs, const uint8_t *__restrict__ done, __nv_bfloat16 *__restrict__ h,
          __nv_bfloat16 *__restrict__ x_out, const float *__restrict__ enc_w,
-         const float *__restrict__ enc_b, int n, int H)
+         const float *__restrict__ enc_b, int n, int H, int chunk_rows, int obs_aligned)
 {
-    const int c = kEncodeCols * threadIdx.x;
-    if (c >= H) return;
-    float w[kEncodeCols][OD], b[kEncodeCols];
-#pragma unroll
-    for (int e = 0; e < kEncodeCols; ++e) {
-        b[e] = __ldg(enc_b + c + e);
-#pragma unroll
-        for (int i = 0; i < OD; ++i) w[e][i] = __ldg(enc_w + static_cast<size_t>(c + e) * OD + i);
-    }
+    constexpr int COLS = EncodeShape<OD>::kCols;
+    extern __shared__ float4 enc_smem[];
+    float *s_obs = reinterpret_cast<float *>(enc_smem + H * (OD + 1) / 4);
+    uint8_t *s_done = reinterpret_cast<uint8_t *>(s_obs + chunk_rows * OD);
     const bool mask = done != nullptr && h != nullptr;
-    for (long long m0 = static_cast<long long>(blockIdx.x) * kEncodeRows; m0 < n;
-         m0 += static_cast<long long>(gridDim.x) * kEncodeRows) {
-        const float *row = obs + static_cast<size_t>(m0) * OD;
-        const uint8_t *done_m0 = mask ? done + m0 : nullptr;
-        __nv_bfloat16 *xrow = x_out + static_cast<size_t>(m0) * H + c;
-        __nv_bfloat16 *hrow = h + static_cast<size_t>(m0) * H + c;
-        if (n - m0 >= kEncodeRows)
-            encode_pass<OD, true>(row, done_m0, hrow, xrow, w, b, kEncodeRows, H);
-        else
-            encode_pass<OD, false>(row, done_m0, hrow, xrow, w, b, static_cast<int>(n - m0), H);
+
+    // the chunk's obs: 16-byte pieces where the source allows (a chunk starts at a multiple of
+    // four envs, so its first byte is 16-byte aligned if obs is), single words otherwise
+    auto stage_chunk = [&](long long r0, int rows) {
+        const float *src = obs + static_cast<size_t>(r0) * OD;
+        const int words = rows * OD;
+        const int vec = obs_aligned ? words / 4 : 0;
+        for (int i = threadIdx.x; i < vec; i += blockDim.x)
+            reinterpret_cast<float4 *>(s_obs)[i] = __ldg(reinterpret_cast<const float4 *>(src) + i);
+        for (int i = 4 * vec + threadIdx.x; i < words; i += blockDim.x) s_obs[i] = __ldg(src + i);
+        for (int i = threadIdx.x; i < chunk_rows; i += blockDim.x)
+            s_done[i] = (mask && i < rows) ? __ldg(done + r0 + i) : 0;
+    };
+
+    {
+        const float4 *gw = reinterpret_cast<const float4 *>(enc_w), *gb = reinterpret_cast<const float4 *>(enc_b);
+        const int nw = H * OD / 4, nb = H / 4;
+        for (int i = threadIdx.x; i < nw; i += blockDim.x) enc_smem[i] = __ldg(gw + i);
+        for (int i = threadIdx.x; i < nb; i += blockDim.x) enc_smem[nw + i] = __ldg(gb + i);
+    }
+    long long r0 = static_cast<long long>(blockIdx.x) * chunk_rows;   // the grid has no more blocks than chunks
+    int rows = static_cast<int>(n - r0 < chunk_rows ? n - r0 : chunk_rows);
+    stage_chunk(r0, rows);
+    __syncthreads();
+
+    const int groups = H / COLS;
+    const int slot = threadIdx.x / groups;
+    const int group = threadIdx.x - slot * groups;
+    const int c = COLS * group;
+    const int slots = blockDim.x / groups;
+    float w[COLS * OD], b[COLS];
+    {
+        const float4 *sw = enc_smem + group * (COLS * OD / 4);
+        const float4 *sb = enc_smem + H * OD / 4 + group * (COLS / 4);
+#pragma unroll
+        for (int i = 0; i < COLS * OD / 4; ++i) {
+            const float4 v = sw[i];
+            w[4 * i] = v.x;
+            w[4 * i + 1] = v.y;
+            w[4 * i + 2] = v.z;
+            w[4 * i + 3] = v.w;
+        }
+#pragma unroll
+        for (int i = 0; i < COLS / 4; ++i) {
+            const float4 v = sb[i];
+            b[4 * i] = v.x;
+            b[4 * i + 1] = v.y;
+            b[4 * i + 2] = v.z;
+            b[4 * i + 3] = v.w;
+        }
+    }
+
+    while (true) {
+        for (int m = slot * kEncodeRows; m < rows; m += slots * kEncodeRows) {
+            const int left = rows - m;   // envs of this pass: kEncodeRows, fewer at the end of the batch
+            float o[kEncodeRows * OD];
+            if (left >= kEncodeRows) {
+#pragma unroll
+                for (int i = 0; i < OD; ++i) {   // m is a multiple of 4: 16-byte aligned in shared memory
+                    const float4 v = reinterpret_cast<const float4 *>(s_obs + m * OD)[i];
+                    o[4 * i] = v.x;
+                    o[4 * i + 1] = v.y;
+                    o[4 * i + 2] = v.z;
+                    o[4 * i + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < kEncodeRows; ++r) {
+                    const int rr = r < left ? r : 0;
+#pragma unroll
+                    for (int i = 0; i < OD; ++i) o[r * OD + i] = s_obs[(m + rr) * OD + i];
+                }
+            }
+            const uint32_t ended = *reinterpret_cast<const uint32_t *>(s_done + m);   // byte r: env m + r
+            __nv_bfloat16 *xrow = x_out + static_cast<size_t>(r0 + m) * H + c;
+#pragma unroll
+            for (int r = 0; r < kEncodeRows; ++r) {
+                if (r >= left) break;
+                // COLS independent chains side by side: no fma waits for the one before it
+                float acc[COLS];
+#pragma unroll
+                for (int e = 0; e < COLS; ++e) acc[e] = b[e];
+#pragma unroll
+                for (int i = 0; i < OD; ++i) {
+#pragma unroll
+                    for (int e = 0; e < COLS; ++e) acc[e] = __fmaf_rn(o[r * OD + i], w[e * OD + i], acc[e]);
+                }
+                uint32_t packed[COLS / 2];
+#pragma unroll
+                for (int e = 0; e < COLS; e += 2) packed[e / 2] = pack_bf16_relu(acc[e], acc[e + 1]);
+                store_units<COLS>(xrow + static_cast<size_t>(r) * H, packed);
+            }
+            if (ended != 0) {   // rare: the cleared units of h
+                uint32_t zero[COLS / 2];
+#pragma unroll
+                for (int e = 0; e < COLS / 2; ++e) zero[e] = 0u;
+                __nv_bfloat16 *hrow = h + static_cast<size_t>(r0 + m) * H + c;
+#pragma unroll
+                for (int r = 0; r < kEncodeRows; ++r)
+                    if ((ended >> (8 * r)) & 0xFFu) store_units<COLS>(hrow + static_cast<size_t>(r) * H, zero);
+            }
+        }
+        r0 += static_cast<long long>(gridDim.x) * chunk_rows;
+        if (r0 >= n) break;
+        rows = static_cast<int>(n - r0 < chunk_rows ? n - r0 : chunk_rows);
+        __syncthreads();   // every slot has read the previous chunk
+        stage_chunk(r0, rows);
+        __syncthreads();
     }
 }
 
+// Threads per block: H/cols unit groups times a slot count: the smallest that fills whole
+// warps, doubled while the block stays within 256 threads; where whole warps would need
+// more than kEncodeMaxThreads, the most slots that fit (the last warp is then partly idle).
+int encode_threads(int H, int cols)
+{
+    const int groups = H / cols;
+    int slots = 1;
+    while ((groups * slots) % 32 != 0) slots *= 2;
+    if (groups * slots > kEncodeMaxThreads) slots = kEncodeMaxThreads / groups;
+    while (groups * slots * 2 <= 256) slots *= 2;
+    return groups * slots;
+}
+
+size_t encode_smem_bytes(int H, int obs_dim, int chunk_rows)
+{
+    return static_cast<size_t>(H) * (obs_dim + 1) * sizeof(float) +
+           static_cast<size_t>(chunk_rows) * (obs_dim * sizeof(float) + 1);
+}
+
 typedef void (*EncodeKernel)(const float *, const uint8_t *, __nv_bfloat16 *, __nv_bfloat16 *, const float *,
-                             const float *, int, int);
+                             const float *, int, int, int, int);
 
 template <int OD>
 struct EncodeTable {
     static EncodeKernel get(int obs_dim) { return obs_dim == OD ? k_encode<OD> : EncodeTable<OD - 1>::get(obs_dim); }
+    static int cols(int obs_dim) { return obs_dim == OD ? EncodeShape<OD>::kCols : EncodeTable<OD - 1>::cols(obs_dim); }
 };
 template <>
 struct EncodeTable<0> {
     static EncodeKernel get(int) { return nullptr; }
+    static int cols(int) { return 4; }
 };
 
 // 64 envs per block, one thread per env.  logits[a] = bias + the partial sums of the blocks of
@@ -978,23 +1078,33 @@ int gru_policy_encode(gru_policy *p, const float *obs, const uint8_t *done, void
     if (n < 1) return GRU_POLICY_EINVAL;
     if ((reinterpret_cast<uintptr_t>(x_out) | reinterpret_cast<uintptr_t>(h)) % 16 != 0) return GRU_POLICY_EALIGN;
     if (reinterpret_cast<uintptr_t>(obs) % 8 != 0) return GRU_POLICY_EALIGN;
-    const unsigned threads = static_cast<unsigned>((p->H / kEncodeCols + 31) / 32 * 32);
+    const int cols = EncodeTable<GRU_POLICY_MAX_OBS>::cols(p->obs_dim);
+    const int threads = encode_threads(p->H, cols);
     EncodeKernel kernel = EncodeTable<GRU_POLICY_MAX_OBS>::get(p->obs_dim);
-    if (p->encode_blocks_per_sm == 0) {   // one full wave of resident blocks: no partial second wave
+    if (p->encode_blocks_per_sm == 0) {   // resident blocks per SM with the largest chunk
+        const size_t most = encode_smem_bytes(p->H, p->obs_dim, kEncodeMaxChunk);
         int per_sm = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, static_cast<int>(threads), 0) != cudaSuccess ||
-            per_sm < 1) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(most)) != cudaSuccess)
+            return GRU_POLICY_ECUDA;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, most) != cudaSuccess || per_sm < 1) {
             cudaGetLastError();
-            per_sm = 4;
+            per_sm = 1;
         }
         p->encode_blocks_per_sm = per_sm;
     }
-    const long long passes = (static_cast<long long>(n) + kEncodeRows - 1) / kEncodeRows;
+    // Chunks of up to kEncodeMaxChunk envs; a batch that one wave of resident blocks can take
+    // in one chunk each is cut into that many chunks (whole passes of the block's slots).
     const long long cap = static_cast<long long>(p->sms) * p->encode_blocks_per_sm;
-    const unsigned blocks = static_cast<unsigned>(passes < cap ? passes : cap);
-    kernel<<<blocks, threads, 0, p->stream>>>(
+    const int rows_per_pass = threads / (p->H / cols) * kEncodeRows;
+    long long chunk = (n + cap - 1) / cap;
+    chunk = (chunk + rows_per_pass - 1) / rows_per_pass * rows_per_pass;
+    if (chunk > kEncodeMaxChunk) chunk = kEncodeMaxChunk;
+    const long long chunks = (n + chunk - 1) / chunk;
+    const unsigned blocks = static_cast<unsigned>(chunks < cap ? chunks : cap);
+    const int obs_aligned = reinterpret_cast<uintptr_t>(obs) % 16 == 0;
+    kernel<<<blocks, static_cast<unsigned>(threads), encode_smem_bytes(p->H, p->obs_dim, static_cast<int>(chunk)), p->stream>>>(
         obs, done, static_cast<__nv_bfloat16 *>(h), static_cast<__nv_bfloat16 *>(x_out), p->enc_w, p->enc_b, n,
-        p->H);
+        p->H, static_cast<int>(chunk), obs_aligned);
     if (cudaGetLastError() != cudaSuccess) return GRU_POLICY_ECUDA;
     p->launches += 1;
     return GRU_POLICY_OK;
