@@ -238,15 +238,31 @@ __device__ __forceinline__ int agent_step(Env &e, int action, int frameskip_rt,
 // warp-uniform votes and commit their results per lane with selects, so the common
 // path is straight-line code.  The frame counter is kept as frames left in the
 // episode (kMaxFrames - len) so that the end test is a compare with zero.
+//
+// With QUEUE, spawns come from a two-entry queue per lane.  A spawn is a pure function
+// of (seed, env, episode, point), and the points of an episode are used in order, so the
+// spawns an env will need next are known in advance: entry 0 is the spawn of its next
+// point in the current episode, entry 1 the one after.  Some lane of a warp scores in
+// about every third step, and a Philox block run for it costs the whole warp as much as
+// one run for all 32 lanes; with the queue the warp runs Philox only when a lane that
+// needs a spawn has none stored (or starts a new episode), and then restocks every
+// lane's queue with the same two blocks.  An entry is 11 bits: vy + 384 (0..768) and,
+// in bit 10, the sign of vx; 0x7FF marks an empty slot.  Without QUEUE every event runs
+// its own Philox block.  Both give the same values; which is faster depends on the launch
+// (see the launcher).
 struct FastEnv {
     int bx, by, vx, vy, apy, opy;
     int sa, so, left, episode, prev;
+    uint32_t spawns;   // entry 0 in bits 0..10, entry 1 in bits 11..21, ones above
 };
+
+constexpr uint32_t kSpawnEmpty = 0x7FFu;
 
 __device__ __forceinline__ void to_fast(FastEnv &f, const Env &e)
 {
     f.bx = e.bx; f.by = e.by; f.vx = e.vx; f.vy = e.vy; f.apy = e.apy; f.opy = e.opy;
     f.sa = e.sa; f.so = e.so; f.left = kMaxFrames - e.len; f.episode = e.episode; f.prev = e.prev;
+    f.spawns = 0xFFFFFFFFu;   // the queue lives within a launch; it starts empty
 }
 
 __device__ __forceinline__ void from_fast(Env &e, const FastEnv &f)
@@ -255,8 +271,18 @@ __device__ __forceinline__ void from_fast(Env &e, const FastEnv &f)
     e.sa = f.sa; e.so = f.so; e.len = kMaxFrames - f.left; e.episode = f.episode; e.prev = f.prev;
 }
 
+// The queue entry of the ball spawned for (episode, point).
+__device__ __forceinline__ uint32_t spawn_entry(uint32_t env_id, uint32_t episode, uint32_t point,
+                                                const RoundKeys &rk)
+{
+    uint32_t o[4];
+    philox4x32_10(point, episode, env_id, 1u, rk, o);
+    return __umulhi(o[1], 769u) | ((o[0] & 1u) << 10);
+}
+
 // Score and / or episode end.  Run by the whole warp when any lane has an event;
 // only lanes with `ev` commit.  `out` says the ball left the court on this lane.
+template <bool QUEUE>
 __device__ __forceinline__ void fast_event(FastEnv &e, bool ev, bool out, uint32_t env_id,
                                            const RoundKeys &rk, Tally &tally, float &reward,
                                            int &done)
@@ -273,13 +299,30 @@ __device__ __forceinline__ void fast_event(FastEnv &e, bool ev, bool out, uint32
     const int episode = e.episode + (dn ? 1 : 0);
     sa = dn ? 0 : sa;
     so = dn ? 0 : so;
-    uint32_t o[4];
-    philox4x32_10((uint32_t)(sa + so), (uint32_t)episode, env_id, 1u, rk, o);
-    const int nvx = (o[0] & 1u) ? kVx0 : -kVx0;
-    const int nvy = (int)__umulhi(o[1], 769u) - kVySpawn;
+    uint32_t ent;   // the spawn of this lane's event, as a queue entry
+    if (QUEUE) {
+        // A new episode makes the stored spawns stale; an empty queue has none.
+        const bool need = ev && (dn || (e.spawns & kSpawnEmpty) == kSpawnEmpty);
+        if (__any_sync(0xffffffffu, need)) {
+            // Restock every lane: a lane with an event takes the spawn of its new point count
+            // now, any other lane will next need the one after its current count.
+            const uint32_t ep = (uint32_t)(ev ? episode : e.episode);
+            const uint32_t point = (uint32_t)(ev ? sa + so : e.sa + e.so + 1);
+            const uint32_t e0 = spawn_entry(env_id, ep, point, rk);
+            const uint32_t e1 = spawn_entry(env_id, ep, point + 1u, rk);
+            e.spawns = e0 | (e1 << 11) | 0xFFC00000u;
+        }
+        ent = e.spawns & kSpawnEmpty;
+        // bit 31 is set: ones move in, the freed slot reads empty
+        if (ev) e.spawns = (uint32_t)((int)e.spawns >> 11);
+    } else {
+        ent = spawn_entry(env_id, (uint32_t)episode, (uint32_t)(sa + so), rk);
+    }
     if (ev) {
         e.sa = sa; e.so = so; e.episode = episode;
-        e.bx = kSpawnBx; e.by = kSpawnBy; e.vx = nvx; e.vy = nvy;
+        e.bx = kSpawnBx; e.by = kSpawnBy;
+        e.vx = (ent & 0x400u) ? kVx0 : -kVx0;
+        e.vy = (int)(ent & 0x3FFu) - kVySpawn;
         reward = r;
         done = dn ? 1 : 0;
         if (dn) { e.left = kMaxFrames; e.apy = kPadY0; e.opy = kPadY0; e.prev = 0; }
@@ -287,6 +330,7 @@ __device__ __forceinline__ void fast_event(FastEnv &e, bool ev, bool out, uint32
 }
 
 // One frame; all 32 lanes of the warp must call it together.
+template <bool QUEUE>
 __device__ __forceinline__ void fast_frame(FastEnv &e, int action, uint32_t env_id,
                                            const RoundKeys &rk, Tally &tally, float &reward,
                                            int &done)
@@ -319,7 +363,7 @@ __device__ __forceinline__ void fast_frame(FastEnv &e, int action, uint32_t env_
     const bool ev = out || e.left == 0;
     reward = 0.f;
     done = 0;
-    if (__any_sync(0xffffffffu, ev)) fast_event(e, ev, out, env_id, rk, tally, reward, done);
+    if (__any_sync(0xffffffffu, ev)) fast_event<QUEUE>(e, ev, out, env_id, rk, tally, reward, done);
 }
 
 // Philox4x32-10 advanced a few rounds at a time, so that the block for the next

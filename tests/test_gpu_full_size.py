@@ -149,3 +149,39 @@ def test_pixel_rollout_16384_envs_T64(torch):
     assert t == launches * T
     for s, o in zip(starts, oras):
         assert state[:, s:s + 24].tobytes() == o.get_state()[0].tobytes()
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_both_event_paths_of_the_tensor_store_kernel(torch, mode):
+    """The tensor-store rollout has two forms of its score / episode-end path and picks by
+    grid size (up to 1.75 waves of resident blocks: spawns from the per-lane queue; above:
+    one Philox block per event).  Every env is compared with the oracle in both: 131,072 envs
+    take the second form, and the same envs run as two handles of 65,536 take the first."""
+    from paper_2603_12145_b200.inputs import random_states
+    n, seed = 131072, 21
+    st = random_states(n, seed=3, near_end=True)
+    ora = oracle.OraclePong(n, seed)
+    ora.set_state(st, 40)
+    expect = [ora.rollout(T, mode) for T in (16, 24)]
+    whole = pong.PongEnv(n, seed)
+    whole.set_state(st, 40)
+    halves = [pong.PongEnv(n // 2, seed, env_id_base=k * (n // 2)) for k in range(2)]
+    for k, hv in enumerate(halves):
+        hv.set_state(np.ascontiguousarray(st[:, k * (n // 2):(k + 1) * (n // 2)]), 40)
+    for (eo, er, ed), T in zip(expect, (16, 24)):
+        go, gr, gd = whole.rollout(T, mode)
+        assert go.cpu().numpy().tobytes() == eo.tobytes()
+        assert gr.cpu().numpy().tobytes() == er.tobytes()
+        assert gd.cpu().numpy().tobytes() == ed.tobytes()
+        for k, hv in enumerate(halves):
+            sl = slice(k * (n // 2), (k + 1) * (n // 2))
+            ho, hr, hd = hv.rollout(T, mode)
+            assert ho.cpu().numpy().tobytes() == np.ascontiguousarray(eo[:, sl]).tobytes()
+            assert hr.cpu().numpy().tobytes() == np.ascontiguousarray(er[:, sl]).tobytes()
+            assert hd.cpu().numpy().tobytes() == np.ascontiguousarray(ed[:, sl]).tobytes()
+    assert int(sum(e[2].sum() for e in expect)) > n // 4          # many episodes ended
+    os_, ot = ora.get_state()
+    gs, gt = whole.get_state()
+    assert gt == ot and gs.tobytes() == os_.tobytes()
+    assert whole.episode_stats() == ora.episode_stats()
+    assert tuple(sum(v) for v in zip(*(hv.episode_stats() for hv in halves))) == ora.episode_stats()
