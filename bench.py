@@ -47,11 +47,11 @@ WORKLOADS = {
     "rollout65k": dict(
         name="fused vector-obs rollout, N=65536 envs, T=128 steps per launch, in-kernel Philox actions",
         n=65536, T=128, mode=0, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 128,
-        kernel="k_rollout_vector_tma", traffic=188.12e6),
+        kernel="k_rollout_vector_tma", traffic=190.17e6),
     "rollout1m": dict(
         name="fused vector-obs rollout, N=1048576 envs, T=32 steps per launch, in-kernel Philox sticky actions",
         n=1048576, T=32, mode=1, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 32,
-        kernel="k_rollout_vector_tma", traffic=982.24e6),
+        kernel="k_rollout_vector_tma", traffic=982.04e6),
     "pixels16k": dict(
         name="pixel-obs rollout, N=16384 envs, T=64 agent steps per launch, frameskip 4, 4-frame ring uint8[N,4,84,84]",
         n=16384, T=64, mode=0, obs_mode=1, frameskip=4, bytes=7056.0 + 5.0 + 64.0 / 64,
