@@ -199,7 +199,7 @@ def policy_oracle_call(n_sample, T, hidden=576):
         for i in range(T):
             x = ogp.encode(obs, p["enc_w"], p["enc_b"])
             h = ogp.bf16_round_f64(ogp.cell(x, h, p["w_ih"], p["w_hh"], p["b_ih"], p["b_hh"]))
-            logits = ogp.head(h, p["head_w"], p["head_b"])
+            logits = ogp.head(h, p["head_w"], p["head_b"]).astype(np.float32)
             obs, _, done = o.step(oracle.sample_actions(logits, words[i]))
             h[done != 0] = 0.0
         state["obs"], state["h"] = obs, h

@@ -17,11 +17,10 @@
  *                                     S7 = -1/5040, S9 = 1/362880
  *   c =       (((C8*z + C6)*z + C4)*z + C2)*z + 1,   C2 = -1/2, C4 = 1/24,
  *                                     C6 = -1/720, C8 = 1/40320
- *   temp     = (force + ((0.05 * (thd*thd)) * s)) * R
- *   thetaacc = (9.8*s - c*temp) / (0.5 * (4/3 - (0.1*(c*c)) * R))
- *   xacc     = temp - ((0.05*thetaacc) * c) * R,      R = binary32(1 / 1.1)
- *   (the constant total mass enters through its pre-computed reciprocal, the
- *   paper's checklist item 8; only the state-dependent denominator is divided by)
+ *   temp     = (force + ((0.05 * (thd*thd)) * s)) / 1.1
+ *   thetaacc = (9.8*s - c*temp) / (0.5 * (4/3 - (0.1*(c*c)) / 1.1))
+ *   xacc     = temp - ((0.05*thetaacc) * c) / 1.1
+ *   (1.1 = total mass; every / is a correctly rounded binary32 division)
  *   x += 0.02*xd; xd += 0.02*xacc; th += 0.02*thd; thd += 0.02*thetaacc
  * (velocities of the step's start move the positions).  Then steps += 1,
  * reward = 1, done = x < -2.4 || x > 2.4 || |th| > 12 degrees || steps >= 500.

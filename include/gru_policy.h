@@ -30,13 +30,16 @@
  *    tensor cores is not specified, so h' is defined up to that: it agrees with
  *    an exact evaluation to within one bfloat16 rounding plus a binary32
  *    accumulation error (see the parity tests for the bound).
- *  - gru_policy_head: binary32.  The hidden units are taken in blocks of 32; a
- *    block's partial sum is a chain of fused multiply-adds from zero over its
- *    units in ascending order; the logit is the bias plus the partial sums added
- *    one by one in block order.  Reproducible bit for bit, so an action sampled
- *    from these logits is decided identically by any implementation that follows
- *    the same order.  gru_policy_cell_head forms the partial sums in the cell's
- *    epilogue, where each block of h' is produced, and gives the same bits.
+ *  - gru_policy_head: the definition logits = W_o h' + b_o, summed in binary32 in
+ *    this library's own order: the hidden units are taken in blocks of 32 (the
+ *    cell kernel's epilogue tile); a block's partial sum is a chain of fused
+ *    multiply-adds from zero over its units in ascending order; the logit is the
+ *    bias plus the partial sums added one by one in block order.  The result is
+ *    within (H + H/32 + 1) * 2^-24 * (|b| + sum |h w|) of the exact value (one
+ *    rounding per fused multiply-add, per partial sum added and for the bias), and
+ *    the same bits on every call.  gru_policy_cell_head forms the partial sums in
+ *    the cell's epilogue, where each block of h' is produced, and gives the bits of
+ *    gru_policy_head applied to its h'.
  *
  * Conventions.  Parameters are given to gru_policy_create as HOST float arrays,
  * rows = output units, gate blocks of w_ih / w_hh / b_ih / b_hh in the order

@@ -21,13 +21,11 @@
  *   z = th*th
  *   s = th * ((((S9*z + S7)*z + S5)*z + S3)*z + 1)          sin(th)
  *   c =       (((C8*z + C6)*z + C4)*z + C2)*z + 1            cos(th)
- *   temp     = (force + ((0.05 * (thd*thd)) * s)) * R
- *   thetaacc = (9.8*s - c*temp) / (0.5 * (4/3 - (0.1*(c*c)) * R))
- *   xacc     = temp - ((0.05*thetaacc) * c) * R
- *   with R = binary32(1 / 1.1): the three divisions by the constant total mass
- *   are multiplications by its pre-computed reciprocal, as the paper's
- *   checklist asks for constant denominators (Appendix "JAX Optimization
- *   Checklist", item 8); the division by the state-dependent denominator stays.
+ *   temp     = (force + ((0.05 * (thd*thd)) * s)) / 1.1
+ *   thetaacc = (9.8*s - c*temp) / (0.5 * (4/3 - (0.1*(c*c)) / 1.1))
+ *   xacc     = temp - ((0.05*thetaacc) * c) / 1.1
+ *   (1.1 = total mass of cart and pole; every / is a correctly rounded binary32
+ *   division, as the textbook equations are written)
  *   x += 0.02*xd;  xd += 0.02*xacc;  th += 0.02*thd;  thd += 0.02*thetaacc
  *   steps += 1;  reward = 1
  *   done = x < -2.4 || x > 2.4 || th < -TH || th > TH || steps >= 500
@@ -62,7 +60,7 @@ typedef struct {
 
 static const float CP_GRAVITY = 9.8f;
 static const float CP_MASSPOLE = 0.1f;
-static const float CP_INV_TOTAL_MASS = 1.0f / 1.1f; /* pre-computed reciprocal, rounded once */
+static const float CP_TOTAL_MASS = 1.1f;    /* cart 1.0 + pole 0.1 */
 static const float CP_LENGTH = 0.5f;        /* half the pole's length */
 static const float CP_POLEMASS_LENGTH = 0.05f;
 static const float CP_FORCE = 10.0f;
@@ -160,21 +158,21 @@ int cp_oracle_step(cp_env *e, int action, uint64_t seed, uint32_t env_id, cp_sta
     float t2 = CP_POLEMASS_LENGTH * t1;
     float t3 = t2 * s;
     float t4 = force + t3;
-    float temp = t4 * CP_INV_TOTAL_MASS;
+    float temp = t4 / CP_TOTAL_MASS;
 
     float n1 = CP_GRAVITY * s;
     float n2 = c * temp;
     float num = n1 - n2;
     float c2 = c * c;
     float d1 = CP_MASSPOLE * c2;
-    float d2 = d1 * CP_INV_TOTAL_MASS;
+    float d2 = d1 / CP_TOTAL_MASS;
     float d3 = CP_FOUR_THIRDS - d2;
     float den = CP_LENGTH * d3;
     float thetaacc = num / den;
 
     float m1 = CP_POLEMASS_LENGTH * thetaacc;
     float m2 = m1 * c;
-    float m3 = m2 * CP_INV_TOTAL_MASS;
+    float m3 = m2 / CP_TOTAL_MASS;
     float xacc = temp - m3;
 
     float dx = CP_TAU * e->xd;

@@ -43,7 +43,7 @@ def lib():
             L.gp_oracle_encode.restype = None
             L.gp_oracle_cell.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp, vp, vp]
             L.gp_oracle_cell.restype = None
-            L.gp_oracle_head.argtypes = [vp, i32, i32, i32, vp, vp, vp]
+            L.gp_oracle_head.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp]
             L.gp_oracle_head.restype = None
             _lib = L
     return _lib
@@ -92,13 +92,14 @@ def cell(x, h, w_ih, w_hh, b_ih, b_hh, with_abs_sum: bool = False):
     return (out, t) if with_abs_sum else out
 
 
-def head(h, head_w, head_b) -> np.ndarray:
-    """float32 [n, A] logits."""
+def head(h, head_w, head_b, with_abs_sum: bool = False):
+    """float64 [n, A] logits W_o h + b_o; with_abs_sum also returns |b_o| + sum |h w| per logit."""
     h, head_w, head_b = _f32(h), _f32(head_w), _f32(head_b)
     n, H = h.shape
     A = head_w.shape[0]
     assert head_w.shape == (A, H) and head_b.shape == (A,)
-    out = np.empty((n, A), dtype=np.float32)
+    out = np.empty((n, A), dtype=np.float64)
+    t = np.empty((n, A), dtype=np.float64) if with_abs_sum else None
     lib().gp_oracle_head(h.ctypes.data, n, H, A, head_w.ctypes.data, head_b.ctypes.data,
-                         out.ctypes.data)
-    return out
+                         out.ctypes.data, t.ctypes.data if with_abs_sum else None)
+    return (out, t) if with_abs_sum else out

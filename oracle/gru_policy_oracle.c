@@ -25,24 +25,25 @@
  *    returns, per output, the sum of the absolute values of the products that
  *    entered its three pre-activations, which is what an accumulation-error
  *    bound scales with.
- *  - The encoder output is rounded to bfloat16 (it is a tensor-core operand)
- *    and the head's logits decide the sampled action, so both are written in
- *    binary32 with one fixed order: the encoder as a chain of fused
- *    multiply-adds starting from the bias, inputs ascending; the head as such
- *    chains over blocks of 32 hidden units, each from zero, whose results are
- *    added to the bias in block order (the block structure lets a device
- *    produce a block's partial sum where the block of hidden units is made).
- *    fmaf and + are correctly rounded, so a second implementation can
- *    reproduce every bit.
+ *  - The encoder output is rounded to bfloat16 (it is a tensor-core operand),
+ *    so it is written in binary32 with one fixed order: a chain of fused
+ *    multiply-adds starting from the bias, inputs ascending.  fmaf is
+ *    correctly rounded, so a second implementation can reproduce every bit.
+ *  - The head is the definition logits = W_o h' + b_o evaluated plainly in
+ *    binary64 (exact products of the binary32 inputs, sums in binary64, bias
+ *    last), like the cell.  It also returns, per logit, |b| + sum |h w|, which
+ *    is what the rounding error of any binary32 summation order scales with;
+ *    a device result is compared within a bound built from it.
  *  - bfloat16 rounding is round-to-nearest-even on the upper 16 bits.
  *
  * One row (env) at a time, plain loops; shares no code with the CUDA path.
  *
  * Pins (tests without a GPU): the cell against torch.nn.GRUCell in binary64
  * on the CPU (a library routine, same definition), closed forms (zero weights,
- * saturated gates keep or replace h), the encoder and head against binary64
- * dot products within their rounding bound, bfloat16 rounding against known
- * bit patterns and ties.
+ * saturated gates keep or replace h), the encoder against binary64 dot
+ * products within its rounding bound, the head against numpy's matrix product
+ * in binary64, exact small-integer cases and one-hot weights, bfloat16
+ * rounding against known bit patterns and ties.
  */
 #include <math.h>
 #include <stddef.h>
@@ -142,24 +143,17 @@ void gp_oracle_cell(const float *x, const float *h, int n, int H, const float *w
     }
 }
 
-/* logits[n][A]: the hidden units are taken in blocks of 32; a block's partial sum is a
- * binary32 fma chain from zero over its units in ascending order; the logit is the bias
- * plus the partial sums, added one by one in block order. */
-enum { GP_HEAD_BLOCK = 32 };
-
+/* logits[n][A] = b_o[a] + sum_k h[k] * W_o[a][k] in binary64; abs_sum[n][A]
+ * (may be NULL) = |b_o[a]| + sum_k |h[k] * W_o[a][k]|. */
 void gp_oracle_head(const float *h, int n, int H, int A, const float *head_w, const float *head_b,
-                    float *logits)
+                    double *logits, double *abs_sum)
 {
     for (int m = 0; m < n; ++m) {
         for (int a = 0; a < A; ++a) {
-            float total = head_b[a];
-            for (int k0 = 0; k0 < H; k0 += GP_HEAD_BLOCK) {
-                float part = 0.0f;
-                for (int k = k0; k < k0 + GP_HEAD_BLOCK && k < H; ++k)
-                    part = fmaf(h[(size_t)m * H + k], head_w[(size_t)a * H + k], part);
-                total = total + part;
-            }
-            logits[(size_t)m * A + a] = total;
+            double t = 0.0;
+            double s = dot64(h + (size_t)m * H, head_w + (size_t)a * H, H, &t);
+            logits[(size_t)m * A + a] = s + (double)head_b[a];
+            if (abs_sum) abs_sum[(size_t)m * A + a] = t + fabs((double)head_b[a]);
         }
     }
 }

@@ -97,13 +97,13 @@ __device__ __forceinline__ void advance(Env &e, int action)
     const float c = __fadd_rn(__fmul_rn(q, z), 1.0f);
 
     const float t3 = __fmul_rn(__fmul_rn(0.05f, __fmul_rn(e.thd, e.thd)), s);
-    const float inv_total = 1.0f / 1.1f;  // reciprocal of the total mass, rounded once
-    const float temp = __fmul_rn(__fadd_rn(force, t3), inv_total);
+    const float total = 1.1f;  // cart 1.0 + pole 0.1
+    const float temp = __fdiv_rn(__fadd_rn(force, t3), total);
     const float num = __fsub_rn(__fmul_rn(9.8f, s), __fmul_rn(c, temp));
-    const float d2 = __fmul_rn(__fmul_rn(0.1f, __fmul_rn(c, c)), inv_total);
+    const float d2 = __fdiv_rn(__fmul_rn(0.1f, __fmul_rn(c, c)), total);
     const float den = __fmul_rn(0.5f, __fsub_rn(4.0f / 3.0f, d2));
     const float thetaacc = __fdiv_rn(num, den);
-    const float m3 = __fmul_rn(__fmul_rn(__fmul_rn(0.05f, thetaacc), c), inv_total);
+    const float m3 = __fdiv_rn(__fmul_rn(__fmul_rn(0.05f, thetaacc), c), total);
     const float xacc = __fsub_rn(temp, m3);
 
     const float dx = __fmul_rn(0.02f, e.xd);

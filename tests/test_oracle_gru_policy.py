@@ -1,7 +1,8 @@
 """Pins of the GRU-policy oracle against things other than itself: torch's
 GRUCell in binary64 (a library routine with the same definition), closed forms,
 one-hot weights that expose a transposed operand or a wrong gate block,
-binary64 dot products with their rounding bounds, bfloat16 bit patterns."""
+binary64 dot products (numpy, exact rationals) with their rounding bounds,
+bfloat16 bit patterns."""
 import numpy as np
 import pytest
 
@@ -157,39 +158,52 @@ def test_encode_against_float64_and_exact_small_integers():
     assert np.array_equal(got, np.maximum(obs_i @ w_i.T + b_i, 0.0))   # |values| <= 57: exact in bf16
 
 
-def test_head_against_float64_and_exact_small_integers():
+def test_head_against_numpy_float64_and_exact_small_integers():
     H, n = 96, 50
     w = policy_weights(H, 11)
     _, h = policy_activations(n, H, 12)
-    got = gp.head(h, w["head_w"], w["head_b"])
+    got, mag = gp.head(h, w["head_w"], w["head_b"], with_abs_sum=True)
+    assert got.dtype == np.float64
     want = h.astype(np.float64) @ w["head_w"].astype(np.float64).T + w["head_b"].astype(np.float64)
-    mag = np.abs(h.astype(np.float64)) @ np.abs(w["head_w"].astype(np.float64)).T + 1.0
-    assert np.all(np.abs(got - want) <= H * 2.0 ** -24 * mag)
+    want_mag = (np.abs(h.astype(np.float64)) @ np.abs(w["head_w"].astype(np.float64)).T
+                + np.abs(w["head_b"].astype(np.float64)))
+    # numpy's product may add in another order: binary64 rounding only
+    assert np.all(np.abs(got - want) <= H * 2.0 ** -52 * want_mag)
+    assert np.allclose(mag, want_mag, rtol=1e-14)
+    # general binary32 values (not only the generated short ones), against exact rationals
+    from fractions import Fraction
     rng = np.random.Generator(np.random.PCG64(13))
+    hg = rng.normal(0, 1, (3, 40)).astype(np.float32)
+    wg = rng.normal(0, 1, (3, 40)).astype(np.float32)
+    bg = rng.normal(0, 1, 3).astype(np.float32)
+    out = gp.head(hg, wg, bg)
+    for m in range(3):
+        for a in range(3):
+            exact = sum(Fraction(float(hg[m, k])) * Fraction(float(wg[a, k])) for k in range(40))
+            exact += Fraction(float(bg[a]))
+            assert abs(Fraction(float(out[m, a])) - exact) <= Fraction(41, 2 ** 52) * 60
     h_i = rng.integers(-4, 5, (n, H)).astype(np.float32)
     w_i = rng.integers(-4, 5, (3, H)).astype(np.float32)
     b_i = rng.integers(-4, 5, 3).astype(np.float32)
-    assert np.array_equal(gp.head(h_i, w_i, b_i), h_i @ w_i.T + b_i)
+    assert np.array_equal(gp.head(h_i, w_i, b_i), (h_i @ w_i.T + b_i).astype(np.float64))
     # a single non-zero weight picks one column: exposes a transposed weight matrix
     w1 = np.zeros((3, H), np.float32); w1[1, 7] = 1.0
     out = gp.head(h, w1, np.zeros(3, np.float32))
     assert np.array_equal(out[:, 1], h[:, 7]) and not out[:, 0].any() and not out[:, 2].any()
+    # the bias belongs to its own logit
+    out = gp.head(np.zeros((2, H), np.float32), w1, np.array([0.25, -1.5, 3.0], np.float32))
+    assert np.array_equal(out, np.array([[0.25, -1.5, 3.0]] * 2))
 
 
-def test_head_block_structure_by_a_case_where_the_order_shows():
-    # unit 0 contributes 2^24; units 32..63 (the second block of 32) contribute 1 each.  Added
-    # one by one to 2^24 every 1 would be rounded away (ties to even); as a block they arrive
-    # as 32, which 2^24 can absorb exactly.
+def test_head_keeps_what_a_binary32_sum_would_lose():
+    # 2^24 from unit 0 plus 33 ones: exact in binary64 whatever the order, whereas a binary32
+    # running sum would drop every 1 added to 2^24 (ties to even)
     H = 64
     h = np.zeros((1, H), np.float32); w = np.zeros((3, H), np.float32)
     h[0, 0] = 4096.0; w[0, 0] = 4096.0
-    h[0, 32:] = 1.0; w[0, 32:] = 1.0
-    w[1, 0] = 4096.0; w[1, 1:33] = 1.0; h[0, 1:32] = 0.0      # row 1: the ones sit across both blocks
+    h[0, 31:] = 1.0; w[0, 31:] = 1.0
     out = gp.head(h, w, np.array([0.0, 0.0, 0.5], np.float32))
-    assert out[0, 0] == 2.0 ** 24 + 32.0
-    # row 1: block 0 holds 2^24 (unit 0) and nothing else that is non-zero in h; block 1 holds unit 32 only
-    assert out[0, 1] == 2.0 ** 24                       # 2^24 + 1 is a tie: to even
-    assert out[0, 2] == 0.5
+    assert out[0, 0] == 2.0 ** 24 + 33.0 and out[0, 1] == 0.0 and out[0, 2] == 0.5
 
 
 def test_generated_parameters_are_bfloat16_representable():
