@@ -65,6 +65,9 @@
  *     aborts, traps or prints.  There is no CPU fallback: without a usable
  *     CUDA device pong_create* fails with PONG_ECUDA.
  *   - A handle is not thread-safe; use one handle per host thread or lock.
+ *     The library also keeps small per-device caches (SM count, the address of
+ *     pong_rollout_static's array) that are filled on first use without a lock:
+ *     make the first call on each device from one thread.
  */
 #ifndef PONG_H_
 #define PONG_H_
@@ -109,19 +112,44 @@ typedef struct {
 
 /* Create n_envs (>= 1) envs on the current CUDA device, in episode 0 at global
  * step 0, on the default stream.  pong_create uses {vector obs, frameskip 1,
- * env_id_base 0}.  Allocates 32 bytes per env of device memory. */
+ * env_id_base 0}.  Allocates 32 bytes per env of device memory: the state of
+ * all envs lives in buffers allocated once, up front (Appendix "JAX Optimization
+ * Checklist", item 7; "Rust Optimization Checklist", item 2), as structure-of-
+ * arrays planes of 32-bit integers (JAX item 6: the smallest type that holds
+ * the values; Rust item 8: one object for all envs on raw buffers). */
 int pong_create(pong_env **out, int n_envs, uint64_t seed);
 int pong_create_ex(pong_env **out, int n_envs, uint64_t seed, const pong_config *cfg);
 
-/* Synchronise the stream and free everything the handle owns.  NULL is OK. */
+/* Synchronise the stream and free everything the handle owns.  NULL is OK.
+ * (Counterpart of pong_create: the only two calls that touch the allocator,
+ * JAX checklist item 7.) */
 int pong_destroy(pong_env *h);
 
 /* Use `cuda_stream` (a cudaStream_t, e.g. torch's current stream) for all
  * later calls; NULL selects the default stream.  The caller orders work
- * across streams. */
+ * across streams.  (The env runs on the learner's device and stream so that
+ * observations never leave the GPU: Sec. 1 and JAX checklist item 4.) */
 int pong_set_stream(pong_env *h, void *cuda_stream);
 
-/* All envs to episode 0, global step 0, statistics cleared.  obs_out may be
+/* Choose the kernel pong_rollout / pong_step use for vector observations: a
+ * tuning and testing knob, results are bit-identical on every path ("do not
+ * change the external behaviour", Appendix "Optimization Agent Prompt").
+ * AUTO picks by batch size.  GENERAL: per-thread stores, any size.  TMA: 64-env
+ * blocks, shared-memory staging, TMA tensor stores.  CHAINS: one block per SM,
+ * warp chains balanced over the SM's schedulers.  A forced path the call does
+ * not qualify for (alignment, T % 8, frameskip, more than 14 x 32 envs per SM)
+ * falls through chains -> tma -> general. */
+#define PONG_PATH_AUTO    0
+#define PONG_PATH_GENERAL 1
+#define PONG_PATH_TMA     2
+#define PONG_PATH_CHAINS  3
+int pong_set_vector_path(pong_env *h, int path);
+
+/* All envs to episode 0, global step 0, statistics cleared (the reset of the
+ * fixed external API: "step, reset, observation and reward shapes stay as they
+ * are", Appendix "Optimization Agent Prompt"; the reset state is a pure
+ * function of (seed, env, episode) so that two backends started from the same
+ * seed can be compared step by step, Sec. 3.2).  obs_out may be
  * NULL; otherwise it receives the initial observation: float32[n][6]
  * (16-byte aligned) or the whole ring uint8[n][4][84][84] (16-byte aligned),
  * all four slots holding the reset frame. */
@@ -153,7 +181,9 @@ int pong_rollout(pong_env *h, int T, int action_mode, const uint8_t *actions,
 int pong_rollout_host(pong_env *h, int T, int action_mode, const uint8_t *actions_host,
                       void *obs_host, float *reward_host, uint8_t *done_host);
 
-/* Write to actions_out (device, uint8[T][n]) the bytes that make
+/* The "matched actions" of the step-level comparison (Sec. 3.2: both backends
+ * are driven by the same seeds and the same action sequence).
+ * Write to actions_out (device, uint8[T][n]) the bytes that make
  * PONG_ACT_EXPLICIT reproduce PONG_ACT_PHILOX (sticky = 0) or
  * PONG_ACT_STICKY (sticky = 1) for global steps t .. t+T-1.  Does not advance
  * the global step. */
@@ -191,14 +221,19 @@ int pong_sample_actions(pong_env *h, const float *logits, const uint32_t *words,
 int pong_get_step_counter(pong_env *h, uint64_t *t);
 int pong_set_step_counter(pong_env *h, uint64_t t);
 
-/* Episodes finished since create / reset / the last clear: their number, the
+/* The episode statistics the paper's Level-4 check compares (Sec. 3.2: episode
+ * returns and lengths of the two backends), reduced on the device.
+ * Episodes finished since create / reset / the last clear: their number, the
  * sum of their returns (agent points - opponent points) and of their lengths
  * in frames.  Exact integers.  Outputs are HOST pointers (any may be NULL).
  * Synchronises the stream. */
 int pong_episode_stats(pong_env *h, int64_t *episodes, int64_t *sum_return,
                        int64_t *sum_length, int clear);
 
-/* Checkpoint / restore.  host_soa is HOST int32[PONG_STATE_FIELDS][n] in the
+/* Checkpoint / restore (the save-state / load-state pair the paper's module
+ * translation keeps for every stateful component, Appendix "Module Translation
+ * Prompt"; it is also what lets a divergence be replayed from the step before).
+ * host_soa is HOST int32[PONG_STATE_FIELDS][n] in the
  * field order named above; t is the global agent step.  set_state validates
  * field ranges (PONG_EINVAL) and leaves statistics untouched.  In pixel mode
  * the ring is the caller's and is not part of the state. */

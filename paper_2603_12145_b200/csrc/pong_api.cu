@@ -22,6 +22,7 @@ struct pong_env {
     long long *stats = nullptr;
     uint64_t t = 0;  // global agent step
     int64_t launches = 0;
+    int vector_path = 0;
     pong::RoundKeys rk;
     // staging for pong_rollout_host, grown on demand
     void *stage = nullptr;
@@ -45,6 +46,7 @@ pong::LaunchArgs base_args(const pong_env *h)
     a.n = h->n;
     a.T = 1;
     a.frameskip = h->cfg.frameskip;
+    a.vector_path = h->vector_path;
     return a;
 }
 
@@ -177,6 +179,14 @@ int pong_set_stream(pong_env *h, void *cuda_stream)
 {
     if (h == nullptr) return PONG_ENULL;
     h->stream = static_cast<cudaStream_t>(cuda_stream);
+    return PONG_OK;
+}
+
+int pong_set_vector_path(pong_env *h, int path)
+{
+    if (h == nullptr) return PONG_ENULL;
+    if (path < PONG_PATH_AUTO || path > PONG_PATH_CHAINS) return PONG_EINVAL;
+    h->vector_path = path;
     return PONG_OK;
 }
 

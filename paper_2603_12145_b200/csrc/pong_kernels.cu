@@ -413,10 +413,270 @@ static bool try_launch_vector_tma(const LaunchArgs &a, cudaStream_t s, cudaError
     return true;
 }
 
+// ---- vector rollout, one block per SM with balanced warp chains ------------------------
+//
+// A warp-step of the rollout costs a scheduler about as many dispatch cycles whatever else
+// runs on it, so a launch whose blocks are all resident from the start takes as long as the
+// scheduler that holds the most warps.  65,536 envs are 13.84 warps per SM: with small blocks
+// two of an SM's four schedulers get four warps, the others three, and the launch runs at
+// the four-warp pace while the store stream would allow more.  Here one 16-warp block per SM
+// owns a contiguous range of up to 14 chains (a chain = 32 consecutive envs, one lane each,
+// with its own two staging buffers and its own TMA tensor stores, so chains never wait for
+// one another).  Warp w sits on scheduler w % 4.  The first 4*floor(c/4) chains stay on
+// warps 0..11 for the whole launch.  When one or two chains are left over, each alternates
+// between two warps on different schedulers (warps 12 and 14, or 13 and 15) every
+// kChainSegment stages, so that over the launch every scheduler carries the same number of
+// chain-steps.  A hand-over is one pass of the env registers through shared memory between
+// two named hardware barriers, each executed exactly once per hand-over by both warps.
+constexpr int kChainMax = 14;                 // chains per block (shared memory)
+constexpr int kChainWarps = 16;
+constexpr int kChainThreads = kChainWarps * 32;
+constexpr int kChainSegment = 2;              // stages a leftover chain runs on one warp
+constexpr int kHandWords = 12;                // FastEnv as 32-bit words
+
+struct ChainStage {
+    float obs[kTmaStage][32 * 6];
+    float reward[kTmaStage][32];
+    uint8_t done[kTmaStage][32];
+};
+static_assert(sizeof(ChainStage) == 7424 && sizeof(ChainStage) % 128 == 0, "stage layout");
+constexpr int kChainSmemBytes = kChainMax * 2 * (int)sizeof(ChainStage) + 2 * kHandWords * 32 * 4 + 128;
+
+__device__ __forceinline__ void named_barrier(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" :: "r"(id), "r"(threads) : "memory");
+}
+
+template <int MODE, bool QUEUE>
+__global__ void __launch_bounds__(kChainThreads, 1)
+k_rollout_vector_chains(const __grid_constant__ LaunchArgs a, const __grid_constant__ VectorMaps maps)
+{
+    extern __shared__ uint8_t chain_smem[];
+    ChainStage *stages;
+    {
+        const uintptr_t base = (reinterpret_cast<uintptr_t>(chain_smem) + 127) & ~(uintptr_t)127;
+        stages = reinterpret_cast<ChainStage *>(base);
+    }
+    uint32_t(*hand)[kHandWords][32] = reinterpret_cast<uint32_t(*)[kHandWords][32]>(stages + kChainMax * 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int groups = (a.n + 31) >> 5;
+    const int g_lo = (int)((long long)blockIdx.x * groups / gridDim.x);
+    const int g_hi = (int)((long long)(blockIdx.x + 1) * groups / gridDim.x);
+    const int c = g_hi - g_lo;          // <= kChainMax (launcher)
+    const int fixed = c & ~3, extra = c & 3;
+    const int S = a.T / kTmaStage;
+
+    // This warp's role: a chain, and which of its segments (runs of seg_len stages) it takes:
+    // first, first + 2, ...  A whole chain is one segment.
+    int chain = -1, seg_len = S, first = 0, slot = 0;
+    if (warp < fixed) {
+        chain = warp;
+    } else if (warp >= 12) {
+        const int k = warp - 12;
+        if ((extra == 1 || extra == 2) && fixed >= 4 && S > kChainSegment) {
+            if ((k & 1) < extra) {
+                slot = k & 1;
+                chain = fixed + slot;
+                seg_len = kChainSegment;
+                first = k >> 1;
+            }
+        } else if (k < extra) {
+            chain = fixed + k;
+        }
+    }
+    if (chain < 0) return;  // whole warps; no block-wide barrier is used anywhere
+    const int segments = (S + seg_len - 1) / seg_len;
+
+    const int n0 = (g_lo + chain) * 32;
+    const bool valid = n0 + lane < a.n;
+    const int n = valid ? n0 + lane : a.n - 1;
+    const uint32_t env_id = a.env_id_base + (uint32_t)n;
+    const size_t act_stride = (size_t)a.n;
+    ChainStage *mine = stages + chain * 2;
+    uint32_t(*h)[32] = hand[slot];
+    Tally tally = {0, 0, 0};
+    FastEnv e;
+
+    for (int j = first; j < segments; j += 2) {
+        const int sa = j * seg_len, sb = min(S, sa + seg_len);
+        // Philox block of the segment's first four steps: independent of the state, so it
+        // runs before the wait for the state
+        unsigned long long g = (a.t0 + (unsigned long long)sa * kTmaStage) >> 2;
+        PhiloxPipe pipe = {0u, 0u, 0u, 0u};
+        if (MODE <= 1) {
+            philox_start(pipe, g, env_id);
+            philox_rounds<0, 10>(pipe, a.rk);
+        }
+        // hand-over j-1 -> j uses barriers in_id (state written) and in_id + 1 (the giver's last
+        // stage buffer has been read by its store); ids alternate with the hand-over's parity
+        const int in_id = 1 + slot * 4 + ((j - 1) & 1) * 2;
+        if (j == 0) {
+            grid_dependency_wait();
+            Env q;
+            load_env(q, a.plane0, a.plane1, n);
+            to_fast(e, q);
+        } else {
+            if (j == 1) grid_dependency_wait();
+            named_barrier(in_id, 64);
+            e.bx = (int)h[0][lane]; e.by = (int)h[1][lane]; e.vx = (int)h[2][lane]; e.vy = (int)h[3][lane];
+            e.apy = (int)h[4][lane]; e.opy = (int)h[5][lane]; e.sa = (int)h[6][lane]; e.so = (int)h[7][lane];
+            e.left = (int)h[8][lane]; e.episode = (int)h[9][lane]; e.prev = (int)h[10][lane];
+            e.spawns = h[11][lane];
+        }
+        const uint8_t *act = MODE == 2 ? a.actions + n + (size_t)sa * kTmaStage * act_stride : nullptr;
+        bool peer_buffer_pending = j > 0;  // the giver's last store may still read buffer (sa+1)&1
+        for (int s = sa; s < sb; ++s) {
+            uint32_t abyte[kTmaStage];
+            if (MODE == 2) {
+#pragma unroll
+                for (int k = 0; k < kTmaStage; ++k) abyte[k] = act[(size_t)k * act_stride];
+                act += (size_t)kTmaStage * act_stride;
+            }
+            if (peer_buffer_pending && s == sa + 1) {
+                named_barrier(in_id + 1, 64);
+                peer_buffer_pending = false;
+            }
+            ChainStage &st = mine[s & 1];
+            // this warp's own store that last read the buffer is the older of its two in flight
+            if (lane == 0) bulk_wait_read<1>();
+            __syncwarp();
+#pragma unroll
+            for (int q = 0; q < kTmaStage / 4; ++q) {
+                const uint32_t w[4] = {pipe.c0, pipe.c1, pipe.c2, pipe.c3};
+                if (MODE <= 1) {
+                    ++g;
+                    philox_start(pipe, g, env_id);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    if (MODE <= 1) {
+                        if (i == 0) philox_rounds<0, 3>(pipe, a.rk);
+                        if (i == 1) philox_rounds<3, 6>(pipe, a.rk);
+                        if (i == 2) philox_rounds<6, 8>(pipe, a.rk);
+                        if (i == 3) philox_rounds<8, 10>(pipe, a.rk);
+                    }
+                    const int k = q * 4 + i;
+                    int action;
+                    if (MODE == 0) action = uniform_action(w[i]);
+                    else if (MODE == 1) action = sticky_repeat(w[i]) ? e.prev : uniform_action(w[i]);
+                    else if (MODE == 2) action = decode_action_byte(abyte[k], e.prev);
+                    else action = a.const_action;
+                    e.prev = action;
+                    float r;
+                    int dn;
+                    fast_frame<QUEUE>(e, action, env_id, a.rk, tally, r, dn);
+                    float2 *o = reinterpret_cast<float2 *>(&st.obs[k][lane * 6]);
+                    o[0] = make_float2(scale_obs(e.bx), scale_obs(e.by));
+                    o[1] = make_float2(scale_obs(e.vx), scale_obs(e.vy));
+                    o[2] = make_float2(scale_obs(e.apy), scale_obs(e.opy));
+                    st.reward[k][lane] = r;
+                    st.done[k][lane] = (uint8_t)dn;
+                }
+            }
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(&maps.obs, &st.obs[0][0], n0 * 3, s * kTmaStage);
+                tma_store_2d(&maps.reward, &st.reward[0][0], n0, s * kTmaStage);
+                tma_store_2d(&maps.done, &st.done[0][0], n0, s * kTmaStage);
+                bulk_commit();
+            }
+        }
+        if (peer_buffer_pending) named_barrier(in_id + 1, 64);  // a segment of a single stage
+
+        if (j + 1 < segments) {
+            // hand over to the other warp of the pair
+            const int out_id = 1 + slot * 4 + (j & 1) * 2;
+            if (lane == 0) bulk_wait_read<1>();  // the next stage's buffer is free
+            h[0][lane] = (uint32_t)e.bx; h[1][lane] = (uint32_t)e.by; h[2][lane] = (uint32_t)e.vx;
+            h[3][lane] = (uint32_t)e.vy; h[4][lane] = (uint32_t)e.apy; h[5][lane] = (uint32_t)e.opy;
+            h[6][lane] = (uint32_t)e.sa; h[7][lane] = (uint32_t)e.so; h[8][lane] = (uint32_t)e.left;
+            h[9][lane] = (uint32_t)e.episode; h[10][lane] = (uint32_t)e.prev; h[11][lane] = e.spawns;
+            __syncwarp();
+            named_barrier(out_id, 64);
+            if (lane == 0) bulk_wait_read<0>();  // and now the last stage's buffer
+            __syncwarp();
+            named_barrier(out_id + 1, 64);
+        } else if (valid) {
+            Env q;
+            from_fast(q, e);
+            store_env(q, a.plane0, a.plane1, n);
+        }
+    }
+    grid_dependency_launch();
+    if (!valid) {
+        tally.episodes = 0;
+        tally.sum_return = 0;
+        tally.sum_length = 0;
+    }
+    flush_tally(tally, a.stats);
+    if (lane == 0) bulk_wait_read<0>();
+}
+
+// Launches the balanced-chains kernel if the call qualifies (see try_launch_vector_tma for
+// the alignment rules; in addition every block must get at most kChainMax chains).  Unless
+// forced, it is taken only where it measured faster than the small-block kernel: 13 or 14
+// chains on the fullest SM, i.e. 56,833 to 66,304 envs on 148 SMs (41.7 against 46.4 us at
+// 65,536 envs, T = 128).  With 12 chains or fewer per SM no scheduler is over-loaded and the
+// small blocks' shared TMA issue (one thread per 64 envs instead of one per 32) wins by 1-3 us.
+static bool try_launch_vector_chains(const LaunchArgs &a, cudaStream_t s, cudaError_t *err, bool forced)
+{
+    if (a.frameskip != 1) return false;
+    if (a.n % 16 != 0 || a.t0 % 4 != 0 || a.T % kTmaStage != 0) return false;
+    const uintptr_t bases = reinterpret_cast<uintptr_t>(a.obs) | reinterpret_cast<uintptr_t>(a.reward) |
+                            reinterpret_cast<uintptr_t>(a.done);
+    if (bases % 16 != 0) return false;
+    const int sms = resident_sm_count();
+    const int groups = (a.n + 31) / 32;
+    const int grid = groups < sms ? groups : sms;
+    const int fullest = (groups + grid - 1) / grid;
+    if (fullest > kChainMax) return false;
+    if (!forced && fullest < 13) return false;
+    TensorMapEncodeFn enc = tensor_map_encoder();
+    if (enc == nullptr) return false;
+    VectorMaps maps;
+    const uint64_t n = (uint64_t)a.n, T = (uint64_t)a.T;
+    if (!encode_rows(enc, &maps.obs, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, a.obs, n * 3, T, n * 24, 96,
+                     kTmaStage) ||
+        !encode_rows(enc, &maps.reward, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.reward, n, T, n * 4, 32,
+                     kTmaStage) ||
+        !encode_rows(enc, &maps.done, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.done, n, T, n, 32, kTmaStage))
+        return false;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kChainThreads);
+    cfg.dynamicSmemBytes = kChainSmemBytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+#define PONG_CHAINS(M)                                                                              \
+    do {                                                                                            \
+        *err = cudaFuncSetAttribute(k_rollout_vector_chains<M, true>,                               \
+                                    cudaFuncAttributeMaxDynamicSharedMemorySize, kChainSmemBytes);  \
+        if (*err == cudaSuccess) *err = cudaLaunchKernelEx(&cfg, k_rollout_vector_chains<M, true>, a, maps); \
+    } while (0)
+    switch (a.action_mode) {
+    case 0: PONG_CHAINS(0); break;
+    case 1: PONG_CHAINS(1); break;
+    case 2: PONG_CHAINS(2); break;
+    default: PONG_CHAINS(3); break;
+    }
+#undef PONG_CHAINS
+    return true;
+}
+
 cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s)
 {
-    cudaError_t tma_err = cudaSuccess;
-    if (try_launch_vector_tma(a, s, &tma_err)) return tma_err != cudaSuccess ? tma_err : cudaGetLastError();
+    cudaError_t fast_err = cudaSuccess;
+    if ((a.vector_path == kPathAuto || a.vector_path == kPathChains) &&
+        try_launch_vector_chains(a, s, &fast_err, a.vector_path == kPathChains))
+        return fast_err != cudaSuccess ? fast_err : cudaGetLastError();
+    if (a.vector_path != kPathGeneral && try_launch_vector_tma(a, s, &fast_err))
+        return fast_err != cudaSuccess ? fast_err : cudaGetLastError();
     const bool full = (a.t0 % 4 == 0) && (a.T % 4 == 0);
     switch (a.action_mode) {
     case 0: launch_vec_mode<0>(a, full, s); break;

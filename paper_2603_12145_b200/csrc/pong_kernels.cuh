@@ -25,7 +25,12 @@ struct LaunchArgs {
     int action_mode;           // 0 Philox, 1 sticky, 2 explicit, 3 constant
     int const_action;          // mode 3
     int frameskip;
+    int vector_path;           // kPath*: which vector-rollout kernel to use
 };
+
+// Vector-rollout kernels (values of pong_set_vector_path).  A forced path that the call
+// does not qualify for falls through: chains -> tma -> general.
+constexpr int kPathAuto = 0, kPathGeneral = 1, kPathTma = 2, kPathChains = 3;
 
 // Each returns the cudaError_t of the launch (cudaGetLastError).
 cudaError_t launch_reset(const LaunchArgs &a, cudaStream_t s);          // state + optional obs / ring

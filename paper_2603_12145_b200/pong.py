@@ -25,7 +25,9 @@ EXPORTS = ("pong_create", "pong_create_ex", "pong_destroy", "pong_set_stream", "
            "pong_step", "pong_rollout", "pong_rollout_host", "pong_fill_actions",
            "pong_episode_stats", "pong_get_state", "pong_set_state", "pong_num_envs",
            "pong_launch_count", "pong_strerror", "pong_rollout_static", "pong_fill_words",
-           "pong_sample_actions", "pong_get_step_counter", "pong_set_step_counter")
+           "pong_sample_actions", "pong_get_step_counter", "pong_set_step_counter",
+           "pong_set_vector_path")
+PATH_AUTO, PATH_GENERAL, PATH_TMA, PATH_CHAINS = 0, 1, 2, 3
 STATIC_MAX_ENVS = 65536
 
 
@@ -65,6 +67,7 @@ def load(build_if_missing: bool = False):
     L.pong_create_ex.argtypes = [ctypes.POINTER(vp), i32, u64, ctypes.POINTER(_Config)]
     L.pong_destroy.argtypes = [vp]
     L.pong_set_stream.argtypes = [vp, vp]
+    L.pong_set_vector_path.argtypes = [vp, i32]
     L.pong_reset.argtypes = [vp, vp]
     L.pong_step.argtypes = [vp, vp, vp, vp, vp]
     L.pong_rollout.argtypes = [vp, i32, i32, vp, vp, vp, vp]
@@ -134,6 +137,10 @@ def pong_destroy(h: int) -> None:
 
 def pong_set_stream(h: int, cuda_stream: int) -> None:
     _check(load().pong_set_stream(h, cuda_stream), "pong_set_stream")
+
+
+def pong_set_vector_path(h: int, path: int) -> None:
+    _check(load().pong_set_vector_path(h, int(path)), "pong_set_vector_path")
 
 
 def pong_reset(h: int, obs_out=None) -> None:
@@ -262,6 +269,9 @@ class PongEnv:
 
     def _stream(self):
         pong_set_stream(self.h, self.torch.cuda.current_stream(self.device).cuda_stream)
+
+    def set_vector_path(self, path: int):
+        pong_set_vector_path(self.h, path)
 
     def close(self):
         if getattr(self, "h", None):

@@ -1,0 +1,105 @@
+"""Parity of the balanced-chains vector rollout (one block per SM, warp chains, leftover
+chains alternating between two warps) with the CPU oracle, element by element, through
+the C ABI with the path forced.  Sizes are chosen so that blocks on a 148-SM part hold
+every mix the kernel distinguishes: one chain, 4 + 1 / 4 + 2 (alternating leftovers),
+4 + 3 (whole leftovers), 8 + 1 / 8 + 2, 12 + 1 / 12 + 2, the largest batch the kernel
+takes, a ragged last chain; stage counts 1, 2, 3 (a last segment of one stage), 5, 16."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2603_12145_b200 import pong
+from paper_2603_12145_b200.inputs import explicit_actions, random_states
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    import torch
+    assert torch.cuda.is_available()
+    pong.load(build_if_missing=True)
+    return torch
+
+
+def same(got, want, what):
+    for g, w, name in zip(got, want, ("obs", "reward", "done")):
+        g = g.cpu().numpy()
+        assert g.shape == w.shape and g.tobytes() == w.tobytes(), "%s: %s differs" % (what, name)
+
+
+def run_pair(env, ora, T, mode, seed):
+    acts = None
+    if mode == pong.ACT_EXPLICIT:
+        acts = explicit_actions(T, env.n, seed=seed, repeat_fraction=0.2, odd_codes=True)
+    elif mode == pong.ACT_CONSTANT:
+        acts = 2
+    got = env.rollout(T, mode, acts if mode != pong.ACT_EXPLICIT else env.torch.from_numpy(acts).cuda())
+    want = ora.rollout(T, mode, acts)
+    return got, want
+
+
+@pytest.mark.parametrize("n,T,mode", [
+    (16, 8, 0), (48, 16, 1), (1040, 24, 2), (4112, 40, 3),
+    (26048, 24, 0), (26048, 40, 1), (33152, 24, 0), (45056, 40, 2),
+    (61568, 16, 0), (65536, 40, 0), (65536, 24, 1), (65536, 16, 2), (66304, 24, 3), (66288, 128, 0),
+])
+def test_chains_path_matches_the_oracle(torch_cuda, n, T, mode):
+    seed, base = 1000 + n % 97, 3
+    env = pong.PongEnv(n, seed, env_id_base=base)
+    env.set_vector_path(pong.PATH_CHAINS)
+    ora = oracle.OraclePong(n, seed, env_id_base=base)
+    for rep in range(2):                       # the second launch starts from the first one's state
+        got, want = run_pair(env, ora, T, mode, seed + rep)
+        same(got, want, "n=%d T=%d mode=%d launch %d" % (n, T, mode, rep))
+    s_gpu, t_gpu = env.get_state()
+    s_cpu, t_cpu = ora.get_state()
+    assert t_gpu == t_cpu and s_gpu.tobytes() == s_cpu.tobytes()
+    assert tuple(env.episode_stats()) == tuple(ora.episode_stats())
+    env.close()
+
+
+def test_chains_path_through_episode_ends(torch_cuda):
+    """Near-end start states: scores at 15-20 and frame counts close to 10,000, so that resets,
+    the step limit and fresh spawn queues fall inside alternating segments."""
+    n, T, seed = 65536, 64, 77
+    env = pong.PongEnv(n, seed)
+    env.set_vector_path(pong.PATH_CHAINS)
+    ora = oracle.OraclePong(n, seed)
+    st = random_states(n, seed, near_end=True)
+    env.set_state(st, 4096)
+    ora.set_state(st, 4096)
+    for mode in (0, 1):
+        got, want = run_pair(env, ora, T, mode, seed)
+        same(got, want, "near-end mode %d" % mode)
+    assert tuple(env.episode_stats()) == tuple(ora.episode_stats())
+    assert env.episode_stats()[0] > n // 2
+    s_gpu, _ = env.get_state()
+    s_cpu, _ = ora.get_state()
+    assert s_gpu.tobytes() == s_cpu.tobytes()
+    env.close()
+
+
+def test_every_path_gives_the_same_bytes_and_unaligned_calls_fall_through(torch_cuda):
+    torch = torch_cuda
+    n, seed = 61440, 5
+    outs = []
+    for path in (pong.PATH_AUTO, pong.PATH_GENERAL, pong.PATH_TMA, pong.PATH_CHAINS):
+        env = pong.PongEnv(n, seed)
+        env.set_vector_path(path)
+        a = env.rollout(16, pong.ACT_PHILOX)      # aligned
+        b = env.rollout(3, pong.ACT_STICKY)       # T % 8 != 0: every path falls through to the general kernel
+        c = env.rollout(13, pong.ACT_PHILOX)      # t0 % 4 != 0
+        outs.append([t.clone() for t in (*a, *b, *c)] + [torch.from_numpy(env.get_state()[0])])
+        env.close()
+    for other in outs[1:]:
+        for x, y in zip(outs[0], other):
+            assert torch.equal(x.cpu(), y.cpu())
+    ora = oracle.OraclePong(n, seed)
+    want = (*ora.rollout(16, 0), *ora.rollout(3, 1), *ora.rollout(13, 0))
+    for g, w in zip(outs[0], want):
+        assert g.cpu().numpy().tobytes() == w.tobytes()
+    with pytest.raises(pong.PongError) as e:
+        env = pong.PongEnv(16, 1)
+        env.set_vector_path(7)
+    assert e.value.code == -1
