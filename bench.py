@@ -12,6 +12,13 @@ statistics reduction, i.e. 8,388,608 env-steps and 243 MB written per step.
                     [--workload rollout65k|rollout1m|pixels16k|step4096|small64|
                                 cartpole65k|cartpole1m|policy65k]
 
+Timing follows the paper's protocol (warm-up excluded, mean and spread over at least
+five runs): a block of K launches (--steps) is repeated, back to back, until at least
+0.25 s of device time and five repeats are in the timed region; `value` comes from the
+whole region, `segments` holds the per-repeat rates, clocks are sampled inside it.
+The default run also appends one short record for each of the other configurations
+("configs").
+
 Prints one JSON line (rank 0).  With --gpus N > 1 it must be launched with
 torchrun, one rank per GPU; each rank simulates its own 65,536 envs (global env
 ids rank*65536 ...), so the scaling is weak and there is no data-path
@@ -256,26 +263,35 @@ def run_reference(args, rank):
     }), flush=True)
 
 
-def run_policy(args, w, rank, world, local):
-    """The policy-in-the-loop workload: K agent steps per CUDA graph replay; a
-    "step" of the benchmark is one replay.  Also times the same graph without the
-    env-side kernels, and the cell kernel alone, to report each part's share."""
+def run_policy(args, w, rank, world, local, full=True):
+    """The policy-in-the-loop workload: K agent steps per CUDA graph replay; a launch of
+    the benchmark is one replay.  full also times the same graph without the env-side
+    kernels and without the policy, to report each part's share, and the end-to-end leg.
+    The cell kernel alone is timed for the tensor roofline either way."""
     import torch
+    import torch.distributed as dist
     from paper_2603_12145_b200 import gru_policy, policy_loop, pong, sharding
     from paper_2603_12145_b200.inputs import policy_weights
     import numpy as np
 
     N, K = w["n"], w["T"]
     hidden = 576
-    steps = args.steps if args.steps > 0 else 100
-    warmup = max(args.warmup, 3)
+    steps = args.steps if (args.steps > 0 and full) else DEFAULT_STEPS["policy65k"]
+    warmup = max(args.warmup, 3) if full else 3
     env_id_base, _ = sharding.shard(rank, world, N)
     gru_policy.load(build_if_missing=True)
     params = policy_weights(hidden, SEED)
     policy = gru_policy.GruPolicy(params, device="cuda:%d" % local)
     n_params = sum(int(np.asarray(v).size) for v in params.values())
-
     parts = max(1, args.parts)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_ranks(x):
+        return sharding.max_over_ranks(x, device="cuda")
 
     def timed(with_env, with_policy=True):
         loop = policy_loop.PipelinedPolicyLoop(N, SEED, policy, K, parts=parts, env_id_base=env_id_base,
@@ -283,30 +299,33 @@ def run_policy(args, w, rank, world, local):
         loop.capture(with_env=with_env, with_policy=with_policy)
         for _ in range(warmup):
             loop.replay()
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        w0 = time.perf_counter()
-        e0.record()
-        for _ in range(steps):
-            loop.replay()
-        e1.record()
-        torch.cuda.synchronize()
+        loop.sync_and_check()
+        per_ms, ms_total, w0, w1 = timed_blocks(loop.replay, steps, barrier, max_ranks,
+                                                min_seconds=args.min_seconds)
+        loop.sync_and_check()
         # launches made while capturing are replayed: count kernels per replay from what a step launches
         per_replay = parts * (K * ((3 if with_policy else 0) + (2 if with_env else 0)) + (1 if with_env else 0))
-        return e0.elapsed_time(e1), w0, time.perf_counter(), loop, steps * per_replay
+        return per_ms, max_ranks(ms_total), w0, w1, loop, len(per_ms) * steps * per_replay
 
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
-    ms_env, w0, w1, loop, launches = timed(True)
-    ms_pol, _, _, _, _ = timed(False)
-    ms_envk, _, _, _, _ = timed(True, with_policy=False)
+    per_ms, ms_env, w0, w1, loop, launches = timed(True)
+    repeats = len(per_ms)
+    replays = repeats * steps
+    clocks = sampler.summary(w0, w1)
+    ms_pol = ms_envk = None
+    if full:
+        p2, ms_pol, _, _, _, _ = timed(False)
+        ms_pol /= len(p2) * steps
+        p3, ms_envk, _, _, _, _ = timed(True, with_policy=False)
+        ms_envk /= len(p3) * steps
     # the cell kernel alone, back to back, all N envs per launch, on operands of the loop's kind
     policy._stream()
     gen = torch.Generator(device="cuda:%d" % local).manual_seed(SEED)
     cx = torch.rand((N, hidden), device="cuda:%d" % local, generator=gen).to(torch.bfloat16)
     ch = (torch.rand((N, hidden), device="cuda:%d" % local, generator=gen) * 2 - 1).to(torch.bfloat16)
     cout = torch.empty_like(ch)
-    cell_reps = K * min(steps, 20)
+    cell_reps = 400 if full else 200
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     for _ in range(3):
         gru_policy.gru_policy_cell(policy.h, cx, ch, cout, N)
@@ -317,16 +336,24 @@ def run_policy(args, w, rank, world, local):
     torch.cuda.synchronize()
     cell_ms = e0.elapsed_time(e1) / cell_reps
     policy.status()
-    # end to end: the step's result (the env's episode statistics) is read back after every replay
-    e2e_steps = max(args.e2e_steps, 1)
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        loop.replay()
-        stats = loop.episode_stats()
-    e2e_s = time.perf_counter() - t0
+    e2e = None
+    stats = loop.episode_stats()
+    if full:
+        # end to end: the step's result (the env's episode statistics) is read back after every replay
+        e2e_steps = max(args.e2e_steps, 1)
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            loop.replay()
+            stats = loop.episode_stats()
+        e2e_s = time.perf_counter() - t0
+        loop.sync_and_check()
+        e2e = {"value": world * e2e_steps * N * K / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 0,
+               "d2h_bytes_per_step": 24, "steps": e2e_steps,
+               "api": "PolicyLoop.replay + read-back of the env's episode statistics"}
     sampler.stop()
-    ms_env = sharding.max_over_ranks(ms_env, device="cuda")
-    value = world * steps * N * K / (ms_env * 1e-3)
+    ms_replay = ms_env / replays
+    value = world * N * K / (ms_replay * 1e-3)
+    seg = spread([steps * N * K / (m * 1e-3) for m in per_ms])
     cell_flops = 2.0 * 6 * hidden * hidden * N          # the six H x H products of one agent step
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
@@ -334,99 +361,113 @@ def run_policy(args, w, rank, world, local):
     except Exception:
         peak_tf, peak_kind = 1400.0, "fallback, sustained"
     achieved_tf = cell_flops / (cell_ms * 1e-3) / 1e12
-    if rank != 0:
-        return
-    # CPU: the whole agent step from the oracles (encoder, binary64 cell, head, sampling, env step)
-    n_s = 64
-    call = policy_oracle_call(n_s, 1, hidden)
-    c0, reps = time.perf_counter(), 0
-    while time.perf_counter() - c0 < max(args.cpu_seconds, 0.2):
-        call()
-        reps += 1
-    cpu_dt = time.perf_counter() - c0
+    roofline = {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
+                "frac": achieved_tf / peak_tf, "peak_source": peak_kind + " cuBLAS bf16",
+                "traffic": None, "kernel": w["kernel"], "kernel_ms": cell_ms,
+                "flops_per_launch": cell_flops,
+                "note": "12 H^2 flops per env: the six H x H products of the GRU cell, timed back "
+                        "to back over all N envs"}
+    del loop, cx, ch, cout
+    policy.close()
+    torch.cuda.empty_cache()
+    if not full:
+        return {"workload_key": "policy65k", "workload": w["name"], "value": value, "unit": UNIT,
+                "us_per_launch": ms_replay * 1e3, "agent_step_us": ms_replay / K * 1e3,
+                "cell_kernel_us": cell_ms * 1e3, "steps": steps, "repeats": repeats,
+                "roofline": roofline, "segments": seg, "clocks": clocks,
+                "dtype": "bf16 policy (f32 accumulate), int32 env", "gpu_launches": int(launches)}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
-        "warmup": warmup, "ms_per_step": ms_env / steps, "higher_is_better": True, "scaling": "weak",
+        "warmup": warmup, "ms_per_step": ms_replay, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 policy (f32 accumulate), int32 env", "data": "synthetic",
+        "repeats": repeats,
         "config": {"workload": w["name"], "workload_key": args.workload, "n_envs_per_gpu": N,
                    "agent_steps_per_graph": K, "policy_parameters": n_params, "hidden": hidden,
                    "parallel_slices": parts,
                    "env_steps_per_step": N * K,
                    "l2": "the policy's activations (226 MB) and weights are read every step; no flush"},
-        "roofline": {"bound": "tensor", "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s",
-                     "frac": achieved_tf / peak_tf, "peak_source": peak_kind + " cuBLAS bf16",
-                     "traffic": None, "kernel": w["kernel"], "kernel_ms": cell_ms,
-                     "flops_per_launch": cell_flops,
-                     "note": "12 H^2 flops per env: the six H x H products of the GRU cell, timed back "
-                             "to back over all N envs"},
-        "agent_step_us": ms_env / steps / K * 1e3,
-        "policy_only_us_per_agent_step": ms_pol / steps / K * 1e3,
-        "env_kernels_only_us_per_agent_step": ms_envk / steps / K * 1e3,
+        "roofline": roofline,
+        "agent_step_us": ms_replay / K * 1e3,
+        "policy_only_us_per_agent_step": ms_pol / K * 1e3,
+        "env_kernels_only_us_per_agent_step": ms_envk / K * 1e3,
         "cell_kernel_us": cell_ms * 1e3,
-        "env_kernels_share_of_step": ms_envk / ms_env,
-        "e2e": {"value": world * e2e_steps * N * K / e2e_s, "unit": UNIT, "h2d_bytes_per_step": 0,
-                "d2h_bytes_per_step": 24, "steps": e2e_steps,
-                "api": "PolicyLoop.replay + read-back of the env's episode statistics"},
+        "env_kernels_share_of_step": ms_envk / ms_replay,
+        "e2e": e2e,
         "gpu_launches": int(launches),
-        "clocks": sampler.summary(w0, w1),
+        "clocks": clocks,
+        "segments": seg,
         "episode_stats": dict(zip(("episodes", "sum_return", "sum_length"), (int(v) for v in stats))),
-        "cpu_baseline": {"value": reps * n_s / cpu_dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "host_cores": os.cpu_count(),
-                         "sample": "whole agent step (encoder, binary64 cell, head, sampling, env step) "
-                                   "of envs 0..%d, %d steps, %.1f s, single thread" % (n_s - 1, reps, cpu_dt)},
     }
-    print(json.dumps(line), flush=True)
+    if rank == 0:
+        # CPU: the whole agent step from the oracles (encoder, binary64 cell, head, sampling, env step)
+        n_s = 64
+        call = policy_oracle_call(n_s, 1, hidden)
+        c0, reps = time.perf_counter(), 0
+        while time.perf_counter() - c0 < max(args.cpu_seconds, 0.2):
+            call()
+            reps += 1
+        cpu_dt = time.perf_counter() - c0
+        line["cpu_baseline"] = {"value": reps * n_s / cpu_dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "host_cores": os.cpu_count(),
+                                "sample": "whole agent step (encoder, binary64 cell, head, sampling, env step) "
+                                          "of envs 0..%d, %d steps, %.1f s, single thread" % (n_s - 1, reps, cpu_dt)}
+    return line
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=0, help="timed launches (default: per workload)")
-    ap.add_argument("--warmup", type=int, default=20)
-    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--workload", default="rollout65k", choices=sorted(WORKLOADS))
-    ap.add_argument("--e2e-steps", type=int, default=8)
-    ap.add_argument("--cpu-seconds", type=float, default=12.0)
-    ap.add_argument("--parts", type=int, default=1,
-                    help="policy65k: independent env slices run as parallel chains of one graph")
-    args = ap.parse_args()
+def timed_blocks(launch, steps, barrier, max_over_ranks, min_seconds=0.25, min_repeats=5, max_repeats=4000):
+    """Times blocks of `steps` launches, back to back, with CUDA events on the launching
+    stream: one untimed block sizes the run, then the block is repeated until the timed
+    work is at least min_seconds and there are at least min_repeats repeats (the paper's
+    protocol: warm-up excluded, mean and spread over N >= 5 runs).  Returns the per-repeat
+    times in ms, the total in ms, and the wall-clock bracket of the timed region."""
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        launch()
+    e1.record()
+    torch.cuda.synchronize()
+    probe_ms = max_over_ranks(e0.elapsed_time(e1))
+    repeats = int(min(max_repeats, max(min_repeats, -(-min_seconds * 1e3 // max(probe_ms, 1e-3)))))
+    barrier()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
+    w0 = time.perf_counter()
+    marks[0].record()
+    for r in range(repeats):
+        for _ in range(steps):
+            launch()
+        marks[r + 1].record()
+    torch.cuda.synchronize()
+    w1 = time.perf_counter()
+    barrier()
+    per = [marks[r].elapsed_time(marks[r + 1]) for r in range(repeats)]
+    return per, marks[0].elapsed_time(marks[-1]), w0, w1
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
 
-    if args.impl == "reference":
-        run_reference(args, rank)
-        return
+def spread(values):
+    mean = sum(values) / len(values)
+    std = (sum((x - mean) ** 2 for x in values) / len(values)) ** 0.5
+    return {"n": len(values), "mean": mean, "std": std, "cv": std / mean if mean else 0.0}
 
+
+DEFAULT_STEPS = {"rollout65k": 200, "rollout1m": 50, "pixels16k": 10, "step4096": 2000,
+                 "cartpole65k": 200, "cartpole1m": 50, "small64": 20, "policy65k": 4}
+
+def run_env(args, key, rank, world, local, full):
+    """One env workload (Pong or CartPole).  full: the run's main workload (adds the
+    end-to-end leg and the CUDA-graph figure's detail); otherwise a short record for the
+    "configs" list.  Returns the JSON-ready dict on every rank."""
     import torch
     import torch.distributed as dist
     from paper_2603_12145_b200 import pong, sharding
     from paper_2603_12145_b200.inputs import explicit_actions
 
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    if world != args.gpus:
-        raise SystemExit("--gpus %d needs torchrun with %d ranks (WORLD_SIZE=%d)" % (
-            args.gpus, args.gpus, world))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    pong.load(build_if_missing=True)
-
-    w = WORKLOADS[args.workload]
-    if w.get("env") == "policy":
-        run_policy(args, w, rank, world, local)
-        return
+    w = WORKLOADS[key]
     N, T, mode = w["n"], w["T"], w["mode"]
     pixels = w["obs_mode"] == 1
     env_steps_per_launch = N * T
     warmup = max(args.warmup, 3)
-    # default launch count: about 0.3 s of timed work
-    default_steps = {"rollout65k": 5000, "rollout1m": 1500, "pixels16k": 200, "step4096": 20000,
-                     "cartpole65k": 5000, "cartpole1m": 1500,
-                     "small64": 300}[args.workload]
-    steps = args.steps if args.steps > 0 else default_steps
+    steps = args.steps if (args.steps > 0 and full) else DEFAULT_STEPS[key]
 
     env_id_base, _ = sharding.shard(rank, world, N)
     is_cartpole = w.get("env") == "cartpole"
@@ -456,7 +497,7 @@ def main():
                   "(launch-latency-bound workload; flushing between launches would time the flush)"
 
     env._stream()
-    if args.workload == "step4096":
+    if key == "step4096":
         # the C entry point itself, with the buffer addresses taken once: the
         # Python wrapper's per-call work would otherwise dominate a 3 us kernel
         ptrs = (acts_d.data_ptr(), obs.data_ptr(), reward.data_ptr(), done.data_ptr())
@@ -472,6 +513,9 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    def max_ranks(x):
+        return sharding.max_over_ranks(x, device="cuda")
+
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
     for _ in range(warmup):
@@ -480,27 +524,15 @@ def main():
         flush.fill_(1)
     barrier()
 
-    # ---- device-resident timing: K launches, CUDA events on the launching stream
-    n_seg = 5 if steps >= 50 else 1
-    marks = [torch.cuda.Event(enable_timing=True) for _ in range(n_seg + 1)]
+    # ---- device-resident timing: repeated blocks of `steps` launches, CUDA events on the launching stream
     launches0 = env.launches
-    w0 = time.perf_counter()
-    marks[0].record()
-    for s in range(n_seg):
-        lo, hi = steps * s // n_seg, steps * (s + 1) // n_seg
-        for _ in range(hi - lo):
-            launch()
-        marks[s + 1].record()
-    torch.cuda.synchronize()
-    w1 = time.perf_counter()
-    launches = env.launches - launches0
-    barrier()
-    ms_total = marks[0].elapsed_time(marks[-1])
-    seg_rates = []
-    for s in range(n_seg):
-        k = steps * (s + 1) // n_seg - steps * s // n_seg
-        seg_rates.append(k * env_steps_per_launch / (marks[s].elapsed_time(marks[s + 1]) * 1e-3))
-    ms_total = sharding.max_over_ranks(ms_total, device="cuda")
+    per_ms, ms_total, w0, w1 = timed_blocks(launch, steps, barrier, max_ranks,
+                                            min_seconds=args.min_seconds)
+    launches = env.launches - launches0 - steps        # without the untimed sizing block
+    repeats = len(per_ms)
+    ms_total = max_ranks(ms_total)
+    seg = spread([steps * env_steps_per_launch / (m * 1e-3) for m in per_ms])
+    clocks = sampler.summary(w0, w1)
     stats = sharding.sum_stats(env.episode_stats(), device="cuda")
 
     # ---- single-step API only: the same launches replayed from a CUDA graph, which
@@ -508,7 +540,7 @@ def main():
     # the env state lives on the device and the host-side step counter (which does
     # not advance on replay) only keys Philox draws and the pixel ring slot.
     graph_info = None
-    if args.workload == "step4096":
+    if key == "step4096":
         per_graph, replays = 100, 50
         side = torch.cuda.Stream()
         side.wait_stream(torch.cuda.current_stream())
@@ -536,73 +568,149 @@ def main():
                       "value": env_steps_per_launch / (g_ms * 1e-3), "unit": UNIT}
 
     # ---- end to end: host buffers in, host buffers out, through pong_rollout_host
-    e2e_steps = max(args.e2e_steps, 1)
-    acts_h = torch.from_numpy(acts_np).pin_memory()
-    obs_h = (torch.zeros((N, 4, 84, 84), dtype=torch.uint8) if pixels
-             else torch.empty((T, N, obs_width), dtype=torch.float32)).pin_memory()
-    rew_h = torch.empty((T, N), dtype=torch.float32).pin_memory()
-    done_h = torch.empty((T, N), dtype=torch.uint8).pin_memory()
-    env._stream()
-    for _ in range(2):
-        rollout_host(env.h, T, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
-    barrier()
-    e0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        rollout_host(env.h, T, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
-    torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - e0
-    e2e_s = sharding.max_over_ranks(e2e_s, device="cuda")
+    e2e = None
+    if full:
+        e2e_steps = max(args.e2e_steps, 1)
+        acts_h = torch.from_numpy(acts_np).pin_memory()
+        obs_h = (torch.zeros((N, 4, 84, 84), dtype=torch.uint8) if pixels
+                 else torch.empty((T, N, obs_width), dtype=torch.float32)).pin_memory()
+        rew_h = torch.empty((T, N), dtype=torch.float32).pin_memory()
+        done_h = torch.empty((T, N), dtype=torch.uint8).pin_memory()
+        env._stream()
+        for _ in range(2):
+            rollout_host(env.h, T, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
+        barrier()
+        e0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            rollout_host(env.h, T, pong.ACT_EXPLICIT, acts_h, obs_h, rew_h, done_h)
+        torch.cuda.synchronize()
+        e2e_s = max_ranks(time.perf_counter() - e0)
+        h2d = acts_h.numel() + (obs_h.numel() if pixels else 0)
+        d2h = obs_h.numel() * obs_h.element_size() + rew_h.numel() * 4 + done_h.numel()
+        e2e = {"value": world * e2e_steps * env_steps_per_launch / e2e_s, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
+               "api": "pong_rollout_host, pinned host buffers, explicit actions"}
     sampler.stop()
     barrier()
 
-    value = world * steps * env_steps_per_launch / (ms_total * 1e-3)
+    total_launches = repeats * steps
+    value = world * total_launches * env_steps_per_launch / (ms_total * 1e-3)
     peak, peak_kind = measured_peak()
-    kernel_ms = ms_total / steps
+    kernel_ms = ms_total / total_launches
     achieved = env_steps_per_launch * w["bytes"] / (kernel_ms * 1e-3) / 1e9
-    h2d = acts_h.numel() + (obs_h.numel() if pixels else 0)
-    d2h = obs_h.numel() * obs_h.element_size() + rew_h.numel() * 4 + done_h.numel()
-
-    if rank == 0:
-        mean = sum(seg_rates) / len(seg_rates)
-        std = (sum((x - mean) ** 2 for x in seg_rates) / len(seg_rates)) ** 0.5
-        line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
-            "warmup": warmup, "ms_per_step": kernel_ms, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32" if is_cartpole else "int32",
-            "data": "synthetic",
-            "config": {
-                "workload": w["name"], "workload_key": args.workload, "n_envs_per_gpu": N, "T": T,
-                "frameskip": w["frameskip"], "seed": SEED, "env_steps_per_step": env_steps_per_launch,
-                "l2": l2_note,
-                "parallelism": "env shards per GPU, no collective" if world > 1 else "single GPU",
-            },
-            "roofline": {
-                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
-                "traffic": w["traffic"],
-                "algorithmic_bytes_per_launch": env_steps_per_launch * w["bytes"],
-                "bytes_per_env_step": w["bytes"],
-                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                "kernel": w["kernel"], "kernel_ms": kernel_ms,
-            },
-            "e2e": {"value": world * e2e_steps * env_steps_per_launch / e2e_s, "unit": UNIT,
-                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": e2e_steps,
-                    "api": "pong_rollout_host, pinned host buffers, explicit actions"},
-            "gpu_launches": int(launches),
-            "clocks": sampler.summary(w0, w1),
-            "segments": {"n": n_seg, "mean": mean, "std": std, "cv": std / mean},
-            "episode_stats": ({"episodes": stats[0], "sum_length": stats[1]} if is_cartpole else
-                              {"episodes": stats[0], "sum_return": stats[1], "sum_length": stats[2]}),
-        }
+    roofline = {
+        "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_source": peak_kind + " copy bandwidth",
+        "traffic": w["traffic"],
+        "algorithmic_bytes_per_launch": env_steps_per_launch * w["bytes"],
+        "bytes_per_env_step": w["bytes"],
+        "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+        "kernel": w["kernel"], "kernel_ms": kernel_ms,
+    }
+    episode_stats = ({"episodes": stats[0], "sum_length": stats[1]} if is_cartpole else
+                     {"episodes": stats[0], "sum_return": stats[1], "sum_length": stats[2]})
+    env.close()
+    del obs, reward, done, flush
+    torch.cuda.empty_cache()
+    if not full:
+        rec = {"workload_key": key, "workload": w["name"], "value": value, "unit": UNIT,
+               "us_per_launch": kernel_ms * 1e3, "steps": steps, "repeats": repeats,
+               "bytes_per_env_step": w["bytes"], "achieved_gbs": achieved,
+               "frac_of_measured": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+               "kernel": w["kernel"], "segments": seg, "clocks": clocks,
+               "dtype": "f32" if is_cartpole else "int32", "gpu_launches": int(launches)}
         if graph_info is not None:
-            line["cuda_graph"] = graph_info
-        if world == 1:
+            rec["cuda_graph"] = graph_info
+        return rec
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": kernel_ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32" if is_cartpole else "int32",
+        "data": "synthetic", "repeats": repeats,
+        "config": {
+            "workload": w["name"], "workload_key": key, "n_envs_per_gpu": N, "T": T,
+            "frameskip": w["frameskip"], "seed": SEED, "env_steps_per_step": env_steps_per_launch,
+            "l2": l2_note,
+            "timing": "%d repeats of a block of %d launches, back to back, CUDA events between "
+                      "blocks; value from the whole timed region, segments = per-repeat rates"
+                      % (repeats, steps),
+            "parallelism": "env shards per GPU, no collective" if world > 1 else "single GPU",
+        },
+        "roofline": roofline,
+        "e2e": e2e,
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "segments": seg,
+        "episode_stats": episode_stats,
+    }
+    if graph_info is not None:
+        line["cuda_graph"] = graph_info
+    return line
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=0,
+                    help="launches per timed block (default: per workload); blocks repeat until "
+                         "--min-seconds of timed work and at least 5 repeats")
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--workload", default="rollout65k", choices=sorted(WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=8)
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--min-seconds", type=float, default=0.25)
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the short records of the other configurations")
+    ap.add_argument("--parts", type=int, default=1,
+                    help="policy65k: independent env slices run as parallel chains of one graph")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2603_12145_b200 import pong
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    if world != args.gpus:
+        raise SystemExit("--gpus %d needs torchrun with %d ranks (WORLD_SIZE=%d)" % (
+            args.gpus, args.gpus, world))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    pong.load(build_if_missing=True)
+
+    w = WORKLOADS[args.workload]
+    if w.get("env") == "policy":
+        line = run_policy(args, w, rank, world, local, full=True)
+    else:
+        line = run_env(args, args.workload, rank, world, local, full=True)
+    # the other configurations, one short record each (single GPU, default workload only)
+    if world == 1 and args.workload == "rollout65k" and not args.no_configs:
+        records = []
+        for key in ("small64", "step4096", "pixels16k", "rollout1m", "cartpole65k", "cartpole1m",
+                    "policy65k"):
+            if WORKLOADS[key].get("env") == "policy":
+                records.append(run_policy(args, WORKLOADS[key], rank, world, local, full=False))
+            else:
+                records.append(run_env(args, key, rank, world, local, full=False))
+        line["configs"] = records
+    if rank == 0:
+        if world == 1 and w.get("env") != "policy":
             rate, reps, dt, n_sample = cpu_oracle_rate(w, args.cpu_seconds)
             line["cpu_baseline"] = {
                 "value": rate, "unit": UNIT, "cores": 1, "kind": "oracle",
                 "host_cores": os.cpu_count(),
                 "sample": "envs 0..%d of the workload, T=%d per call, %d calls, %.1f s, "
-                          "single thread" % (n_sample - 1, T, reps, dt)}
+                          "single thread" % (n_sample - 1, w["T"], reps, dt)}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

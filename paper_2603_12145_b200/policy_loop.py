@@ -111,12 +111,21 @@ class PolicyLoop:
         self.with_env = with_env
 
     def replay(self):
-        """K more agent steps from the captured graph."""
+        """K more agent steps from the captured graph.  Enqueues only: the results are valid
+        once sync_and_check() (or policy.status()) has returned without raising."""
         if self.with_env:
             pong.pong_fill_words(self.env.h, self.K, self.words)
         self.graph.replay()
         if self.with_env:
             self.env.t = self.env.t + self.K
+
+    def sync_and_check(self):
+        """Synchronises the policy's stream and raises GruPolicyError (ETIMEOUT) if a cell
+        kernel since the last check gave up a bounded wait: its h' and logits, and everything
+        the env did with them, are then invalid.  The error word belongs to the policy handle,
+        so loops that share a policy share it; whoever checks first sees (and clears) it."""
+        self._streams()
+        self.policy.status()
 
 
 class PipelinedPolicyLoop:
@@ -179,6 +188,7 @@ class PipelinedPolicyLoop:
         self.with_env = with_env
 
     def replay(self):
+        """K more agent steps of every slice.  Enqueues only: see sync_and_check()."""
         if self.with_env:
             for part in self.parts:
                 part._streams()
@@ -187,6 +197,13 @@ class PipelinedPolicyLoop:
         if self.with_env:
             for part in self.parts:
                 part.env.t = part.env.t + self.K
+
+    def sync_and_check(self):
+        """Synchronises the device and raises if any slice's cell kernel gave up a wait (one
+        error word for all slices: it says that some result since the last check is invalid)."""
+        self.torch.cuda.synchronize(self.device)
+        self.parts[0]._streams()
+        self.policy.status()
 
     def episode_stats(self):
         totals = [0, 0, 0]
