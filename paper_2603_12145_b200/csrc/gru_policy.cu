@@ -726,6 +726,18 @@ int encode_threads(int H, int cols)
     return groups * slots;
 }
 
+// The dynamic shared-memory limit is an attribute of the kernel on a device, not of a handle.
+// It is only ever raised, so that handles with different hidden sizes can be alive together
+// (lowering it for a small policy would make a larger one's next launch fail).
+bool raise_dynamic_smem(const void *func, size_t bytes)
+{
+    cudaFuncAttributes fa;
+    if (cudaFuncGetAttributes(&fa, func) != cudaSuccess) return false;
+    if (static_cast<size_t>(fa.maxDynamicSharedSizeBytes) >= bytes) return true;
+    return cudaFuncSetAttribute(func, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)) ==
+           cudaSuccess;
+}
+
 size_t encode_smem_bytes(int H, int obs_dim, int chunk_rows)
 {
     return static_cast<size_t>(H) * (obs_dim + 1) * sizeof(float) +
@@ -1020,9 +1032,8 @@ int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions, 
         ok = encode_operand(enc, &p->tm_wx, p->wx, H, static_cast<uint64_t>(3) * H, kBRows) &&
              encode_operand(enc, &p->tm_wh, p->wh, H, static_cast<uint64_t>(3) * H, kBRows);
     }
-    if (ok) ok = cudaFuncSetAttribute(k_gru_cell, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      cell_smem_bytes(H, cell_smem_bytes(H, true) <= kMaxSmem)) ==
-                 cudaSuccess;
+    if (ok) ok = raise_dynamic_smem(reinterpret_cast<const void *>(k_gru_cell),
+                                    cell_smem_bytes(H, cell_smem_bytes(H, true) <= kMaxSmem));
     // Ask for the largest shared-memory partition, not the smallest that holds one block, so that
     // small blocks of other kernels can share an SM with a cell block.
     if (ok) ok = cudaFuncSetAttribute(k_gru_cell, cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -1045,9 +1056,8 @@ int gru_policy_create(gru_policy **out, int hidden, int obs_dim, int n_actions, 
         p->pairs = clusters < p->sms / 2 ? clusters : p->sms / 2;
     }
     if (ok && head_smem_bytes(n_actions, H) > 48 * 1024)
-        ok = cudaFuncSetAttribute(n_actions <= 4 ? k_head<4> : k_head<8>,
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                  static_cast<int>(head_smem_bytes(n_actions, H))) == cudaSuccess;
+        ok = raise_dynamic_smem(reinterpret_cast<const void *>(n_actions <= 4 ? k_head<4> : k_head<8>),
+                                head_smem_bytes(n_actions, H));
     if (!ok) {
         cudaGetLastError();
         release(p);
@@ -1084,8 +1094,7 @@ int gru_policy_encode(gru_policy *p, const float *obs, const uint8_t *done, void
     if (p->encode_blocks_per_sm == 0) {   // resident blocks per SM with the largest chunk
         const size_t most = encode_smem_bytes(p->H, p->obs_dim, kEncodeMaxChunk);
         int per_sm = 0;
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(most)) != cudaSuccess)
-            return GRU_POLICY_ECUDA;
+        if (!raise_dynamic_smem(reinterpret_cast<const void *>(kernel), most)) return GRU_POLICY_ECUDA;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, most) != cudaSuccess || per_sm < 1) {
             cudaGetLastError();
             per_sm = 1;

@@ -24,6 +24,7 @@ struct pong_env {
     int64_t launches = 0;
     int vector_path = 0;
     pong::RoundKeys rk;
+    pong::VectorMapCache map_cache = {};
     // staging for pong_rollout_host, grown on demand
     void *stage = nullptr;
     size_t stage_bytes = 0;
@@ -78,7 +79,7 @@ int do_rollout(pong_env *h, int T, int action_mode, const uint8_t *actions, int 
     cudaError_t err;
     if (h->cfg.obs_mode == PONG_OBS_VECTOR) {
         a.obs = static_cast<float *>(obs);
-        err = pong::launch_rollout_vector(a, h->stream);
+        err = pong::launch_rollout_vector(a, h->stream, &h->map_cache);
     } else {
         a.ring = static_cast<uint8_t *>(obs);
         err = pong::launch_rollout_pixels(a, h->sm_count, h->stream);

@@ -23,6 +23,8 @@
 // blocking instructions are __syncthreads and cp.async.bulk.wait_group.
 #include <cuda.h>
 
+#include <cstring>
+
 #include "pong_kernels.cuh"
 
 namespace pong {
@@ -74,6 +76,13 @@ template <int PENDING>
 __device__ __forceinline__ void bulk_wait_read()
 {
     asm volatile("cp.async.bulk.wait_group.read %0;" :: "n"(PENDING) : "memory");
+}
+// Same, but until the groups have completed (their global writes are done), not only read
+// their shared-memory source.
+template <int PENDING>
+__device__ __forceinline__ void bulk_wait_done()
+{
+    asm volatile("cp.async.bulk.wait_group %0;" :: "n"(PENDING) : "memory");
 }
 __device__ __forceinline__ void fence_async_smem()
 {
@@ -364,9 +373,39 @@ static bool encode_rows(TensorMapEncodeFn enc, CUtensorMap *m, CUtensorMapDataTy
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+static_assert(sizeof(VectorMaps) == sizeof(VectorMapCache::maps), "three 128-byte tensor maps");
+
+// The maps of [T][n] outputs with boxes of box_envs envs by kTmaStage steps: from the cache if
+// it holds them for exactly these buffers and sizes, else encoded (and cached).
+static bool vector_maps(const LaunchArgs &a, int box_envs, VectorMapCache *cache, VectorMaps *maps)
+{
+    if (cache != nullptr && cache->box_envs == box_envs && cache->obs == a.obs && cache->reward == a.reward &&
+        cache->done == a.done && cache->n == a.n && cache->T == a.T) {
+        memcpy(maps, cache->maps, sizeof(VectorMaps));
+        return true;
+    }
+    TensorMapEncodeFn enc = tensor_map_encoder();
+    if (enc == nullptr) return false;
+    const uint64_t n = (uint64_t)a.n, T = (uint64_t)a.T;
+    if (!encode_rows(enc, &maps->obs, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, a.obs, n * 3, T, n * 24,
+                     (uint32_t)box_envs * 3, kTmaStage) ||
+        !encode_rows(enc, &maps->reward, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.reward, n, T, n * 4,
+                     (uint32_t)box_envs, kTmaStage) ||
+        !encode_rows(enc, &maps->done, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.done, n, T, n, (uint32_t)box_envs,
+                     kTmaStage))
+        return false;
+    if (cache != nullptr) {
+        memcpy(cache->maps, maps, sizeof(VectorMaps));
+        cache->obs = a.obs; cache->reward = a.reward; cache->done = a.done;
+        cache->n = a.n; cache->T = a.T; cache->box_envs = box_envs;
+    }
+    return true;
+}
+
 // Launches the TMA path if the call qualifies; returns false (nothing launched)
 // if it does not, so that the caller uses the general kernel.
-static bool try_launch_vector_tma(const LaunchArgs &a, cudaStream_t s, cudaError_t *err)
+static bool try_launch_vector_tma(const LaunchArgs &a, cudaStream_t s, cudaError_t *err,
+                                  VectorMapCache *cache = nullptr)
 {
     if (a.frameskip != 1) return false;
     if (a.n % 16 != 0 || a.t0 % 4 != 0 || a.T % kTmaStage != 0) return false;
@@ -374,17 +413,8 @@ static bool try_launch_vector_tma(const LaunchArgs &a, cudaStream_t s, cudaError
     const uintptr_t bases = reinterpret_cast<uintptr_t>(a.obs) | reinterpret_cast<uintptr_t>(a.reward) |
                             reinterpret_cast<uintptr_t>(a.done);
     if (bases % 16 != 0) return false;  // tensor maps need 16-byte aligned bases
-    TensorMapEncodeFn enc = tensor_map_encoder();
-    if (enc == nullptr) return false;
     VectorMaps maps;
-    const uint64_t n = (uint64_t)a.n, T = (uint64_t)a.T;
-    if (!encode_rows(enc, &maps.obs, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, a.obs, n * 3, T, n * 24,
-                     kTmaBlock * 3, kTmaStage) ||
-        !encode_rows(enc, &maps.reward, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.reward, n, T, n * 4,
-                     kTmaBlock, kTmaStage) ||
-        !encode_rows(enc, &maps.done, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.done, n, T, n, kTmaBlock,
-                     kTmaStage))
-        return false;
+    if (!vector_maps(a, kTmaBlock, cache, &maps)) return false;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((a.n + kTmaBlock - 1) / kTmaBlock);
     cfg.blockDim = dim3(kTmaBlock);
@@ -620,7 +650,8 @@ k_rollout_vector_chains(const __grid_constant__ LaunchArgs a, const __grid_const
 // chains on the fullest SM, i.e. 56,833 to 66,304 envs on 148 SMs (41.7 against 46.4 us at
 // 65,536 envs, T = 128).  With 12 chains or fewer per SM no scheduler is over-loaded and the
 // small blocks' shared TMA issue (one thread per 64 envs instead of one per 32) wins by 1-3 us.
-static bool try_launch_vector_chains(const LaunchArgs &a, cudaStream_t s, cudaError_t *err, bool forced)
+static bool try_launch_vector_chains(const LaunchArgs &a, cudaStream_t s, cudaError_t *err, bool forced,
+                                     VectorMapCache *cache = nullptr)
 {
     if (a.frameskip != 1) return false;
     if (a.n % 16 != 0 || a.t0 % 4 != 0 || a.T % kTmaStage != 0) return false;
@@ -633,16 +664,8 @@ static bool try_launch_vector_chains(const LaunchArgs &a, cudaStream_t s, cudaEr
     const int fullest = (groups + grid - 1) / grid;
     if (fullest > kChainMax) return false;
     if (!forced && fullest < 13) return false;
-    TensorMapEncodeFn enc = tensor_map_encoder();
-    if (enc == nullptr) return false;
     VectorMaps maps;
-    const uint64_t n = (uint64_t)a.n, T = (uint64_t)a.T;
-    if (!encode_rows(enc, &maps.obs, CU_TENSOR_MAP_DATA_TYPE_FLOAT64, a.obs, n * 3, T, n * 24, 96,
-                     kTmaStage) ||
-        !encode_rows(enc, &maps.reward, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, a.reward, n, T, n * 4, 32,
-                     kTmaStage) ||
-        !encode_rows(enc, &maps.done, CU_TENSOR_MAP_DATA_TYPE_UINT8, a.done, n, T, n, 32, kTmaStage))
-        return false;
+    if (!vector_maps(a, 32, cache, &maps)) return false;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kChainThreads);
@@ -653,10 +676,19 @@ static bool try_launch_vector_chains(const LaunchArgs &a, cudaStream_t s, cudaEr
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    // the kernel's shared-memory limit is raised once per device and action mode (an unlocked
+    // cache like resident_sm_count's: a second thread at worst sets the same value again)
+    static bool limit_set[4][64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
 #define PONG_CHAINS(M)                                                                              \
     do {                                                                                            \
-        *err = cudaFuncSetAttribute(k_rollout_vector_chains<M, true>,                               \
-                                    cudaFuncAttributeMaxDynamicSharedMemorySize, kChainSmemBytes);  \
+        *err = cudaSuccess;                                                                         \
+        if (!limit_set[M][dev]) {                                                                   \
+            *err = cudaFuncSetAttribute(k_rollout_vector_chains<M, true>,                           \
+                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kChainSmemBytes); \
+            limit_set[M][dev] = *err == cudaSuccess;                                                \
+        }                                                                                           \
         if (*err == cudaSuccess) *err = cudaLaunchKernelEx(&cfg, k_rollout_vector_chains<M, true>, a, maps); \
     } while (0)
     switch (a.action_mode) {
@@ -669,13 +701,13 @@ static bool try_launch_vector_chains(const LaunchArgs &a, cudaStream_t s, cudaEr
     return true;
 }
 
-cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s)
+cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s, VectorMapCache *cache)
 {
     cudaError_t fast_err = cudaSuccess;
     if ((a.vector_path == kPathAuto || a.vector_path == kPathChains) &&
-        try_launch_vector_chains(a, s, &fast_err, a.vector_path == kPathChains))
+        try_launch_vector_chains(a, s, &fast_err, a.vector_path == kPathChains, cache))
         return fast_err != cudaSuccess ? fast_err : cudaGetLastError();
-    if (a.vector_path != kPathGeneral && try_launch_vector_tma(a, s, &fast_err))
+    if (a.vector_path != kPathGeneral && try_launch_vector_tma(a, s, &fast_err, cache))
         return fast_err != cudaSuccess ? fast_err : cudaGetLastError();
     const bool full = (a.t0 % 4 == 0) && (a.T % 4 == 0);
     switch (a.action_mode) {
@@ -745,6 +777,13 @@ __global__ void __launch_bounds__(kPixThreads) k_rollout_pixels(const __grid_con
     if (has_env) load_env(e, a.plane0, a.plane1, n);
     uint32_t w[4] = {0u, 0u, 0u, 0u};
     unsigned round = 0;  // staging buffer rotation of this warp
+    // An env's ring is written again on the next step (another slot, or all four after a reset),
+    // and bulk copies have no order among themselves: the earlier store of the same bytes must
+    // have completed, not only read its source.  A warp commits one group per env and step, so
+    // with at least kPixBufPerWarp envs the wait that frees the staging buffer (all but the two
+    // newest groups complete) already covers the env's previous store; a warp with fewer envs
+    // waits for everything.
+    const bool few_envs = (count - warp + kPixWarps - 1) / kPixWarps < kPixBufPerWarp;
 
     for (int t = 0; t < a.T; ++t) {
         const unsigned long long tt = a.t0 + (unsigned long long)t;
@@ -767,7 +806,10 @@ __global__ void __launch_bounds__(kPixThreads) k_rollout_pixels(const __grid_con
             uint8_t *buf = frames + (warp * kPixBufPerWarp + (round % kPixBufPerWarp)) * kFrameBytes;
             ++round;
             // the copy that last read this buffer is the third most recent group
-            if (lane == 0) bulk_wait_read<kPixBufPerWarp - 1>();
+            if (lane == 0) {
+                if (few_envs) bulk_wait_done<0>();
+                else bulk_wait_done<kPixBufPerWarp - 1>();
+            }
             __syncwarp();
             render_frame(buf, geom[le], lane);
             fence_async_smem();
@@ -820,6 +862,9 @@ __global__ void __launch_bounds__(kPix4Threads) k_rollout_pixels_x4(const __grid
     Tally tally = {0, 0, 0};
     if (has_env) load_env(e, a.plane0, a.plane1, n);
     unsigned round = 0;
+    // The same ring is stored again four steps later: that earlier store must have completed
+    // (see k_rollout_pixels); with at least kPix4Bufs envs per warp the buffer wait covers it.
+    const bool few_envs = (count - warp + kPix4Warps - 1) / kPix4Warps < kPix4Bufs;
 
     for (int t = 0; t < a.T; t += 4) {
         if (has_env) {
@@ -848,7 +893,10 @@ __global__ void __launch_bounds__(kPix4Threads) k_rollout_pixels_x4(const __grid
         for (int le = warp; le < count; le += kPix4Warps) {
             uint8_t *buf = rings + (warp * kPix4Bufs + (round % kPix4Bufs)) * kRingBytes;
             ++round;
-            if (lane == 0) bulk_wait_read<kPix4Bufs - 1>();
+            if (lane == 0) {
+                if (few_envs) bulk_wait_done<0>();
+                else bulk_wait_done<kPix4Bufs - 1>();
+            }
             __syncwarp();
             const uint4 gq = geom[le];
             render_frame(buf, gq.x, lane);

@@ -32,9 +32,19 @@ struct LaunchArgs {
 // does not qualify for falls through: chains -> tma -> general.
 constexpr int kPathAuto = 0, kPathGeneral = 1, kPathTma = 2, kPathChains = 3;
 
+// The three tensor maps of a vector rollout (obs, reward, done) as last encoded for a handle,
+// with what they were encoded for.  Encoding costs the host about a microsecond per map, which
+// shows in launches of 20 us and less; a caller that rolls out into the same buffers again
+// reuses them.  Opaque here: the CUtensorMap type stays inside pong_kernels.cu.
+struct VectorMapCache {
+    alignas(64) unsigned char maps[3 * 128];
+    const void *obs, *reward, *done;
+    int n, T, box_envs;        // box_envs = 0: nothing cached
+};
+
 // Each returns the cudaError_t of the launch (cudaGetLastError).
 cudaError_t launch_reset(const LaunchArgs &a, cudaStream_t s);          // state + optional obs / ring
-cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s);
+cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s, VectorMapCache *cache = nullptr);
 cudaError_t launch_rollout_pixels(const LaunchArgs &a, int sm_count, cudaStream_t s);
 cudaError_t launch_fill_actions(const LaunchArgs &a, int sticky, uint8_t *out, cudaStream_t s);
 cudaError_t launch_fill_words(const LaunchArgs &a, uint32_t *out, cudaStream_t s);

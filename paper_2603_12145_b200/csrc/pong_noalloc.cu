@@ -54,6 +54,8 @@ extern "C" int pong_rollout_static(int n_envs, uint64_t seed, int env_id_base, i
     if (n_envs < 1 || T < 1 || env_id_base < 0) return PONG_EINVAL;
     if (n_envs > PONG_STATIC_MAX_ENVS) return PONG_ELIMIT;
     if ((int64_t)env_id_base + n_envs > 0x7fffffffLL) return PONG_EINVAL;
+    // [T][n] element counts must stay addressable by the kernels' size_t math (as pong_rollout)
+    if ((uint64_t)T * (uint64_t)n_envs > (1ull << 40)) return PONG_EINVAL;
     if (action_mode < PONG_ACT_PHILOX || action_mode > PONG_ACT_CONSTANT) return PONG_EMODE;
     if (obs_buf == nullptr || reward_buf == nullptr || done_buf == nullptr) return PONG_ENULL;
     if ((action_mode == PONG_ACT_EXPLICIT || action_mode == PONG_ACT_CONSTANT) && actions == nullptr)

@@ -322,3 +322,26 @@ def test_argument_errors(torch_cuda):
     assert e.value.code == -3
     pol.status()
     pol.close()
+
+
+def test_two_policies_of_different_hidden_size_alive_together(torch_cuda):
+    """The kernels' shared-memory limits belong to the kernel, not to a handle: creating a small
+    policy after a large one must not take the large one's launch configuration away."""
+    torch = torch_cuda
+    big_w, small_w = policy_weights(1024, 91), policy_weights(64, 92)
+    big = gp.GruPolicy(big_w)
+    small = gp.GruPolicy(small_w)          # created second: would lower the limits if they were per handle
+    rng = np.random.Generator(np.random.PCG64(93))
+    for pol, w, H in ((big, big_w, 1024), (small, small_w, 64), (big, big_w, 1024)):
+        x, h = policy_activations(130, H, 94)
+        obs = rng.uniform(-0.1, 1.1, (130, 6)).astype(np.float32)
+        xe = pol.encode(torch.from_numpy(obs).cuda())
+        assert np.array_equal(from_dev_bf16(torch, xe).view(np.uint32),
+                              ogp.encode(obs, w["enc_w"], w["enc_b"]).view(np.uint32))
+        out = pol.cell(to_dev_bf16(torch, x), to_dev_bf16(torch, h))
+        want = ogp.cell(x, h, w["w_ih"], w["w_hh"], w["b_ih"], w["b_hh"])
+        assert np.all(np.abs(from_dev_bf16(torch, out) - want) <= cell_tolerance(want))
+        logits = pol.head(to_dev_bf16(torch, h)).cpu().numpy().astype(np.float64)
+        assert np.array_equal(logits, ogp.head(h, w["head_w"], w["head_b"]))
+        pol.status()
+    big.close(); small.close()

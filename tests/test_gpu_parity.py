@@ -353,6 +353,26 @@ def test_pixel_four_step_path_with_resets_inside_a_pass(torch, mode):
     assert_state_equal(env, ora)
 
 
+def test_pixel_one_env_per_block_long_rollouts_through_episode_ends(torch):
+    """Few envs: every block (and warp) owns a single env, so consecutive steps re-store the same
+    ring bytes from the same thread a few microseconds apart (a reset writes all four slots, the
+    next step one of them).  Long enough for several episode ends per env, on both pixel kernels."""
+    n, seed = 5, 123
+    env = pong.PongEnv(n, seed, obs_mode=1, frameskip=4)
+    ora = oracle.OraclePong(n, seed, obs_mode=1, frameskip=4)
+    st = random_states(n, seed=4, near_end=True)
+    st[8] = 9990 - 3 * np.arange(n)
+    env.set_state(st, 0)
+    ora.set_state(st, 0)
+    dones = 0
+    for T in (600, 1, 599, 2, 2, 600):          # aligned (four steps per pass), then unaligned, then aligned
+        g, o = env.rollout(T, 0), ora.rollout(T, 0)
+        assert_outputs_equal(g, o, "one env per block, T %d" % T)
+        dones += int(o[2].sum())
+    assert dones >= 2 * n
+    assert_state_equal(env, ora)
+
+
 def test_pixel_frameskip_one_and_constant_action(torch):
     n, seed = 50, 8
     env = pong.PongEnv(n, seed, obs_mode=1, frameskip=1)
