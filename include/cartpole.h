@@ -92,8 +92,10 @@ int cartpole_rollout_host(cartpole_env *h, int T, int action_mode, const uint8_t
 int cartpole_episode_stats(cartpole_env *h, int64_t *episodes, int64_t *sum_length, int clear);
 
 /* Checkpoint / restore: HOST float32[4][n] = x, xd, th, thd; HOST int32[2][n] =
- * steps, episode; t = global step.  set_state rejects NaN / infinite values,
- * steps outside 0..499 and negative episodes. */
+ * steps, episode; t = global step.  set_state accepts in-play states only
+ * (|x| <= 2.4, |th| <= 12 degrees: an env never rests in a state that ends its
+ * episode) with |xd|, |thd| <= 1000, steps in 0..499 and episode >= 0; anything
+ * else, NaN included, is CARTPOLE_EINVAL. */
 int cartpole_get_state(cartpole_env *h, float *host_f, int32_t *host_i, uint64_t *t);
 int cartpole_set_state(cartpole_env *h, const float *host_f, const int32_t *host_i, uint64_t t);
 

@@ -113,6 +113,50 @@ def test_step_limit_truncation_with_balancing_actions(torch):
     assert_state_equal(env, ora)
 
 
+def test_extreme_in_play_states_divide_exactly(torch):
+    """The kernel forms x / 1.1 by a multiply and two fused steps, which equals the division the
+    oracle performs except for |x| <= 3.39e-32 and -0.  States at the edges of what set_state
+    accepts (zero, signed-zero, subnormal and tiny angles, velocities up to +-1000, and angular
+    velocities chosen so that force + 0.05 thd^2 sin(th) cancels to zero or to one ulp) must
+    still agree with the oracle bit for bit."""
+    th_vals = np.array([0.0, -0.0, 1e-45, -1e-45, 1e-38, -1e-38, 1e-30, 3e-20, -3e-20, 1e-7, -1e-7,
+                        0.05, -0.05, 0.2094, -0.2094, 0.20943951], np.float32)
+    thd_vals = np.array([0.0, -0.0, 1e-38, 1e-20, -1e-20, 1.0, -1.0, 30.9, -30.9, 63.2, 100.0, -100.0,
+                         999.0, -999.0, 1000.0, -1000.0], np.float32)
+    th, thd = np.meshgrid(th_vals, thd_vals, indexing="ij")
+    th, thd = th.ravel(), thd.ravel()
+    # rows where t3 = 0.05 thd^2 sin(th) lands on -+10 exactly or within a few ulps: solve for thd
+    extra_th = np.array([0.2, -0.2, 0.1, -0.1, 0.01, -0.01] * 40, np.float32)
+    target = np.float32(10.0)
+    base = np.sqrt(np.float64(target) / (0.05 * np.abs(np.sin(np.float64(extra_th))))).astype(np.float32)
+    extra_thd = base.view(np.uint32) + np.tile(np.arange(-20, 20, dtype=np.int64).repeat(6), 1)[:len(base)]
+    extra_thd = extra_thd.astype(np.uint32).view(np.float32)
+    th = np.concatenate([th, extra_th])
+    thd = np.concatenate([thd, extra_thd])
+    keep = np.abs(thd) <= 1000.0
+    th, thd = th[keep], thd[keep]
+    n = len(th)
+    rng = np.random.Generator(np.random.PCG64(8))
+    f = np.stack([rng.uniform(-2.3, 2.3, n).astype(np.float32), rng.uniform(-50, 50, n).astype(np.float32),
+                  th, thd])
+    i = np.zeros((2, n), np.int32)
+    for action in (0, 1):
+        env, ora = cp.CartPoleEnv(n, 3), ocp.OracleCartPole(n, 3)
+        env.set_state(f, i, 0)
+        ora.set_state(f, i, 0)
+        for t in range(3):
+            g = env.rollout(1, cp.ACT_CONSTANT, action)
+            o = ora.rollout(1, 3, action)
+            assert_equal(g, o, "extreme states, action %d step %d" % (action, t))
+        assert_state_equal(env, ora)
+    # states outside the accepted range are refused
+    for k, v in ((0, 2.5), (1, 1001.0), (2, 0.21), (3, -1000.5), (3, np.inf)):
+        bad = f.copy(); bad[k, 0] = v
+        with pytest.raises(cp.CartPoleError) as ei:
+            env.set_state(bad, i, 0)
+        assert ei.value.code == -1
+
+
 def test_state_roundtrip_restore_partition_and_errors(torch):
     seed = 5
     whole = cp.CartPoleEnv(96, seed)
