@@ -3,7 +3,8 @@ chains alternating between two warps) with the CPU oracle, element by element, t
 the C ABI with the path forced.  Sizes are chosen so that blocks on a 148-SM part hold
 every mix the kernel distinguishes: one chain, 4 + 1 / 4 + 2 (alternating leftovers),
 4 + 3 (whole leftovers), 8 + 1 / 8 + 2, 12 + 1 / 12 + 2, the largest batch the kernel
-takes, a ragged last chain; stage counts 1, 2, 3 (a last segment of one stage), 5, 16."""
+takes, a ragged last chain; stage counts 1, 2, 3 (no alternation), 5 and 9 (a last segment of one
+stage), 6, 8, 16."""
 import numpy as np
 import pytest
 
@@ -41,8 +42,8 @@ def run_pair(env, ora, T, mode, seed):
 
 @pytest.mark.parametrize("n,T,mode", [
     (16, 8, 0), (48, 16, 1), (1040, 24, 2), (4112, 40, 3),
-    (26048, 24, 0), (26048, 40, 1), (33152, 24, 0), (45056, 40, 2),
-    (61568, 16, 0), (65536, 40, 0), (65536, 24, 1), (65536, 16, 2), (66304, 24, 3), (66288, 128, 0),
+    (26048, 24, 0), (26048, 40, 1), (26048, 72, 0), (33152, 24, 0), (45056, 40, 2), (45056, 64, 1),
+    (61568, 16, 0), (65536, 40, 0), (65536, 72, 1), (65536, 48, 2), (66304, 64, 3), (66288, 128, 0),
 ])
 def test_chains_path_matches_the_oracle(torch_cuda, n, T, mode):
     seed, base = 1000 + n % 97, 3
