@@ -49,16 +49,20 @@ FALLBACK_HBM_GBS = 6650.0
 # 32-byte state read and written once per launch (64 / T); the single-step API
 # also reads one action byte.  CartPole: obs 16 + reward 4 + done 1, state 24 bytes.
 # traffic: dram__bytes_read.sum + dram__bytes_write.sum of one launch from an ncu
-# capture of that workload (profiles/), None if not captured for the current kernel.
+# capture of that workload (profiles/; for the two vector rollouts a steady-state capture
+# without cache flushes), None if not captured for the current kernel.
+# alu_per_warp_step: integer-ALU-pipe instructions the kernel executes per warp and agent
+# step, from the same profiles (sm__inst_executed_pipe_alu); with the ALU rate measured live
+# it gives the secondary, compute-side ceiling of the rollout.
 WORKLOADS = {
     "rollout65k": dict(
         name="fused vector-obs rollout, N=65536 envs, T=128 steps per launch, in-kernel Philox actions",
         n=65536, T=128, mode=0, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 128,
-        kernel="k_rollout_vector_tma", traffic=190.17e6),
+        kernel="k_rollout_vector_chains", traffic=244.07e6, alu_per_warp_step=55.5),
     "rollout1m": dict(
         name="fused vector-obs rollout, N=1048576 envs, T=32 steps per launch, in-kernel Philox sticky actions",
         n=1048576, T=32, mode=1, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 32,
-        kernel="k_rollout_vector_tma", traffic=982.04e6),
+        kernel="k_rollout_vector_tma", traffic=1038.9e6, alu_per_warp_step=44.5),
     "pixels16k": dict(
         name="pixel-obs rollout, N=16384 envs, T=64 agent steps per launch, frameskip 4, 4-frame ring uint8[N,4,84,84]",
         n=16384, T=64, mode=0, obs_mode=1, frameskip=4, bytes=7056.0 + 5.0 + 64.0 / 64,
@@ -607,6 +611,17 @@ def run_env(args, key, rank, world, local, full):
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "kernel": w["kernel"], "kernel_ms": kernel_ms,
     }
+    if w.get("alu_per_warp_step"):
+        # secondary ceiling: what the integer pipe alone would allow.  Rate measured now on this
+        # device (register-only add / max / min chains at full occupancy), instruction count per
+        # warp-step from the kernel's ncu profile.
+        alu_rate = pong.pong_measure_alu_rate(torch.cuda.current_stream().cuda_stream)
+        ceiling = alu_rate / w["alu_per_warp_step"] * 32.0
+        roofline["secondary"] = {
+            "bound": "alu", "unit": UNIT, "ceiling": ceiling, "frac": value / world / ceiling,
+            "alu_warp_instr_per_s": alu_rate, "alu_instr_per_warp_step": w["alu_per_warp_step"],
+            "note": "integer-ALU rate measured live (pong_measure_alu_rate) / ALU instructions per "
+                    "warp-step from the ncu profile of this kernel x 32 envs per warp"}
     episode_stats = ({"episodes": stats[0], "sum_length": stats[1]} if is_cartpole else
                      {"episodes": stats[0], "sum_return": stats[1], "sum_length": stats[2]})
     env.close()
@@ -619,6 +634,8 @@ def run_env(args, key, rank, world, local, full):
                "frac_of_measured": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                "kernel": w["kernel"], "segments": seg, "clocks": clocks,
                "dtype": "f32" if is_cartpole else "int32", "gpu_launches": int(launches)}
+        if "secondary" in roofline:
+            rec["secondary"] = roofline["secondary"]
         if graph_info is not None:
             rec["cuda_graph"] = graph_info
         return rec

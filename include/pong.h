@@ -273,6 +273,14 @@ int pong_rollout_static(int n_envs, uint64_t seed, int env_id_base, int T, int a
                         const uint8_t *actions, float *obs_buf, float *reward_buf,
                         uint8_t *done_buf, int64_t *stats_out, void *cuda_stream);
 
+/* Measurement aid for the compute-side ceiling of the rollout (the paper's optimisation
+ * loop profiles before it optimises, Sec. 3.3; a kernel that is all integer min / max / add
+ * has the integer pipe as its second roofline next to HBM): runs a register-only kernel of
+ * dependent add / max / min chains at full occupancy on the current device and returns the
+ * integer-ALU warp instructions per second it sustained (HOST double).  Synchronises
+ * cuda_stream.  Allocates nothing. */
+int pong_measure_alu_rate(void *cuda_stream, double *warp_instr_per_s);
+
 /* Number of envs / kernels launched by this handle so far (for accounting). */
 int pong_num_envs(const pong_env *h);
 int64_t pong_launch_count(const pong_env *h);

@@ -395,6 +395,15 @@ int pong_set_state(pong_env *h, const int32_t *s, uint64_t t)
     return PONG_OK;
 }
 
+int pong_measure_alu_rate(void *cuda_stream, double *warp_instr_per_s)
+{
+    if (warp_instr_per_s == nullptr) return PONG_ENULL;
+    *warp_instr_per_s = 0.0;
+    return pong::measure_alu_rate(static_cast<cudaStream_t>(cuda_stream), warp_instr_per_s) == cudaSuccess
+               ? PONG_OK
+               : PONG_ECUDA;
+}
+
 int pong_num_envs(const pong_env *h) { return h ? h->n : PONG_ENULL; }
 
 int64_t pong_launch_count(const pong_env *h) { return h ? h->launches : (int64_t)PONG_ENULL; }

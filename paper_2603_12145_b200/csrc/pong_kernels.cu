@@ -1105,4 +1105,67 @@ cudaError_t launch_sample_actions(int n, const float *logits, const uint32_t *wo
     return cudaGetLastError();
 }
 
+// ---- integer-ALU rate probe ----------------------------------------------------------------
+//
+// The rollout is integer min / max / add / compare / select work; on sm_100a those run on
+// the half-rate ALU pipe of each scheduler.  This kernel measures what that pipe sustains:
+// every thread runs kAluChains independent chains of max / xor / min / xor on registers,
+// long enough and at full occupancy, so that the time is
+// the pipe's and not latency.  Used by the benchmark for the secondary (compute) ceiling.
+constexpr int kAluChains = 8;
+constexpr int kAluOpsPerIter = kAluChains * 4;  // max, xor, min, xor per chain
+
+__device__ int g_alu_sink;
+
+__global__ void __launch_bounds__(256) k_alu_probe(const int iters, const int seed)
+{
+    int v[kAluChains];
+#pragma unroll
+    for (int c = 0; c < kAluChains; ++c) v[c] = seed + (int)threadIdx.x * (c + 1);
+    int d = (int)(threadIdx.x & 7) - 3;
+    for (int i = 0; i < iters; ++i) {
+#pragma unroll
+        for (int c = 0; c < kAluChains; ++c) {
+            // four dependent ALU-pipe operations; a logic operation between the min and the max
+            // keeps the assembler from merging neighbours into one three-input instruction
+            asm volatile("max.s32 %0, %0, %2;\n\txor.b32 %0, %0, %1;\n\tmin.s32 %0, %0, %3;\n\txor.b32 %0, %0, %1;"
+                         : "+r"(v[c]) : "r"(d), "r"(c), "r"(kPadYMax + c));
+        }
+    }
+    int acc = 0;
+#pragma unroll
+    for (int c = 0; c < kAluChains; ++c) acc ^= v[c];
+    if (acc == 0x7fffffff) g_alu_sink = acc;  // keeps the chains alive; never true in practice
+}
+
+cudaError_t measure_alu_rate(cudaStream_t s, double *warp_instr_per_s)
+{
+    int dev = 0, sms = 0;
+    cudaError_t err = cudaGetDevice(&dev);
+    if (err == cudaSuccess) err = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (err != cudaSuccess) return err;
+    const int blocks = sms * 8, threads = 256, iters = 4096;  // 64 warps per SM
+    cudaEvent_t e0, e1;
+    if ((err = cudaEventCreate(&e0)) != cudaSuccess) return err;
+    if ((err = cudaEventCreate(&e1)) != cudaSuccess) { cudaEventDestroy(e0); return err; }
+    k_alu_probe<<<blocks, threads, 0, s>>>(64, 1);  // warm-up
+    float best = 0.f;
+    for (int rep = 0; rep < 5 && err == cudaSuccess; ++rep) {
+        cudaEventRecord(e0, s);
+        k_alu_probe<<<blocks, threads, 0, s>>>(iters, rep);
+        cudaEventRecord(e1, s);
+        err = cudaEventSynchronize(e1);
+        float ms = 0.f;
+        if (err == cudaSuccess) err = cudaEventElapsedTime(&ms, e0, e1);
+        if (err == cudaSuccess && (best == 0.f || ms < best)) best = ms;
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (err != cudaSuccess) return err;
+    if ((err = cudaGetLastError()) != cudaSuccess) return err;
+    const double warp_instr = (double)blocks * (threads / 32) * (double)iters * kAluOpsPerIter;
+    *warp_instr_per_s = warp_instr / ((double)best * 1e-3);
+    return cudaSuccess;
+}
+
 }  // namespace pong

@@ -51,4 +51,7 @@ cudaError_t launch_fill_words(const LaunchArgs &a, uint32_t *out, cudaStream_t s
 cudaError_t launch_sample_actions(int n, const float *logits, const uint32_t *words, uint8_t *out,
                                   cudaStream_t s);
 
+// Integer-ALU warp instructions per second the device sustains (synchronises the stream).
+cudaError_t measure_alu_rate(cudaStream_t s, double *warp_instr_per_s);
+
 }  // namespace pong

@@ -26,7 +26,7 @@ EXPORTS = ("pong_create", "pong_create_ex", "pong_destroy", "pong_set_stream", "
            "pong_episode_stats", "pong_get_state", "pong_set_state", "pong_num_envs",
            "pong_launch_count", "pong_strerror", "pong_rollout_static", "pong_fill_words",
            "pong_sample_actions", "pong_get_step_counter", "pong_set_step_counter",
-           "pong_set_vector_path")
+           "pong_set_vector_path", "pong_measure_alu_rate")
 PATH_AUTO, PATH_GENERAL, PATH_TMA, PATH_CHAINS = 0, 1, 2, 3
 STATIC_MAX_ENVS = 65536
 
@@ -68,6 +68,7 @@ def load(build_if_missing: bool = False):
     L.pong_destroy.argtypes = [vp]
     L.pong_set_stream.argtypes = [vp, vp]
     L.pong_set_vector_path.argtypes = [vp, i32]
+    L.pong_measure_alu_rate.argtypes = [vp, ctypes.POINTER(ctypes.c_double)]
     L.pong_reset.argtypes = [vp, vp]
     L.pong_step.argtypes = [vp, vp, vp, vp, vp]
     L.pong_rollout.argtypes = [vp, i32, i32, vp, vp, vp, vp]
@@ -141,6 +142,13 @@ def pong_set_stream(h: int, cuda_stream: int) -> None:
 
 def pong_set_vector_path(h: int, path: int) -> None:
     _check(load().pong_set_vector_path(h, int(path)), "pong_set_vector_path")
+
+
+def pong_measure_alu_rate(cuda_stream: Optional[int] = None) -> float:
+    """Integer-ALU warp instructions per second the current device sustains."""
+    out = ctypes.c_double(0.0)
+    _check(load().pong_measure_alu_rate(cuda_stream, ctypes.byref(out)), "pong_measure_alu_rate")
+    return out.value
 
 
 def pong_reset(h: int, obs_out=None) -> None:
