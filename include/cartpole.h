@@ -99,6 +99,15 @@ int cartpole_episode_stats(cartpole_env *h, int64_t *episodes, int64_t *sum_leng
 int cartpole_get_state(cartpole_env *h, float *host_f, int32_t *host_i, uint64_t *t);
 int cartpole_set_state(cartpole_env *h, const float *host_f, const int32_t *host_i, uint64_t t);
 
+/* Which rollout kernel runs (a tuning / testing knob; every path gives the same bits).
+ * AUTO picks by batch size.  PLAIN: 128-env blocks.  CHAINS: one block per SM with its warps'
+ * load balanced over the SM's schedulers; needs the global step and T to be multiples of 4 and
+ * at most 14 x 32 envs per SM, otherwise the plain kernel runs. */
+#define CARTPOLE_PATH_AUTO   0
+#define CARTPOLE_PATH_PLAIN  1
+#define CARTPOLE_PATH_CHAINS 2
+int cartpole_set_path(cartpole_env *h, int path);
+
 int cartpole_num_envs(const cartpole_env *h);
 int64_t cartpole_launch_count(const cartpole_env *h);
 const char *cartpole_strerror(int code);

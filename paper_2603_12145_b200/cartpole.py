@@ -16,7 +16,8 @@ ACT_PHILOX, ACT_EXPLICIT, ACT_CONSTANT = 0, 2, 3
 EXPORTS = ("cartpole_create", "cartpole_destroy", "cartpole_set_stream", "cartpole_reset",
            "cartpole_step", "cartpole_rollout", "cartpole_rollout_host", "cartpole_episode_stats",
            "cartpole_get_state", "cartpole_set_state", "cartpole_num_envs",
-           "cartpole_launch_count", "cartpole_strerror")
+           "cartpole_launch_count", "cartpole_strerror", "cartpole_set_path")
+PATH_AUTO, PATH_PLAIN, PATH_CHAINS = 0, 1, 2
 
 
 class CartPoleError(RuntimeError):
@@ -51,6 +52,7 @@ def load(build_if_missing: bool = False):
     L.cartpole_get_state.argtypes = [vp, vp, vp, ctypes.POINTER(u64)]
     L.cartpole_set_state.argtypes = [vp, vp, vp, u64]
     L.cartpole_num_envs.argtypes = [vp]
+    L.cartpole_set_path.argtypes = [vp, i32]
     L.cartpole_launch_count.argtypes = [vp]
     L.cartpole_launch_count.restype = i64
     L.cartpole_strerror.argtypes = [i32]
@@ -148,6 +150,10 @@ def cartpole_set_state(h: int, fstate, istate, t: int) -> None:
     _check(load().cartpole_set_state(h, f.ctypes.data, i.ctypes.data, int(t)), "cartpole_set_state")
 
 
+def cartpole_set_path(h: int, path: int) -> None:
+    _check(load().cartpole_set_path(h, int(path)), "cartpole_set_path")
+
+
 def cartpole_num_envs(h: int) -> int:
     return int(load().cartpole_num_envs(h))
 
@@ -221,6 +227,9 @@ class CartPoleEnv:
     def get_state(self):
         self._stream()
         return cartpole_get_state(self.h)
+
+    def set_path(self, path: int):
+        cartpole_set_path(self.h, path)
 
     def set_state(self, fstate, istate, t):
         self._stream()

@@ -182,8 +182,61 @@ __global__ void __launch_bounds__(kBlock) k_cartpole_reset(const __grid_constant
 constexpr int kChunk = 128;
 constexpr int kTable = 1 + (kChunk - 1) / 8;
 
+// Steps [c0, c1) of one env (c1 - c0 <= kChunk): fills the thread's table column (entries
+// column[k * pitch]) with the start states of its next episodes, then steps.  The output
+// pointers are those of step c0 and are advanced.
 // MODE 0: Philox actions (one block of four words serves four steps), 2: explicit
-// bytes, 3: constant.  FULL: t0 and T are multiples of 4.
+// bytes, 3: constant.  FULL: c0 and c1 are multiples of 4.
+template <int MODE, bool FULL>
+__device__ __forceinline__ void run_span(Env &e, const uint32_t env_id, const unsigned long long c0,
+                                         const unsigned long long c1, float4 *column, const int pitch,
+                                         float4 *&obs, float *&rew, uint8_t *&dn, const uint8_t *&act,
+                                         const size_t stride, int &episodes, int &sum_length, const Args &a)
+{
+    const int filled = 1 + ((int)(c1 - c0) - 1) / 8;
+    for (int k = 0; k < filled; ++k) {
+        Env r;
+        reset_env(r, env_id, (uint32_t)(e.episode + 1 + k), a.rk);
+        column[k * pitch] = make_float4(r.x, r.xd, r.th, r.thd);
+    }
+    int used = 0;
+    for (unsigned long long g = c0 >> 2; g <= (c1 - 1) >> 2; ++g) {
+        uint32_t w[4] = {0u, 0u, 0u, 0u};
+        if (MODE == 0) philox((uint32_t)g, env_id, (uint32_t)(g >> 32), 3u, a.rk, w);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const unsigned long long tt = g * 4 + j;
+            if (FULL || (tt >= c0 && tt < c1)) {
+                int action;
+                if (MODE == 0) action = (int)(w[j] & 1u);
+                else if (MODE == 2) { action = *act & 1u; act += stride; }
+                else action = a.const_action;
+                advance(e, action);
+                const bool done = terminated(e);
+                if (done) {
+                    episodes += 1;
+                    sum_length += e.steps;
+                    e.episode += 1;
+                    e.steps = 0;
+                    if (used < filled) {
+                        const float4 r = column[used * pitch];
+                        e.x = r.x; e.xd = r.y; e.th = r.z; e.thd = r.w;
+                        used += 1;
+                    } else {
+                        reset_env(e, env_id, (uint32_t)e.episode, a.rk);
+                    }
+                }
+                *obs = make_float4(e.x, e.xd, e.th, e.thd);
+                *rew = 1.0f;
+                *dn = done ? 1 : 0;
+                obs += stride;
+                rew += stride;
+                dn += stride;
+            }
+        }
+    }
+}
+
 template <int MODE, bool FULL>
 __global__ void __launch_bounds__(kBlock) k_cartpole_rollout(const __grid_constant__ Args a)
 {
@@ -206,54 +259,116 @@ __global__ void __launch_bounds__(kBlock) k_cartpole_rollout(const __grid_consta
         uint8_t *dn = a.done + n;
         const uint8_t *act = MODE == 2 ? a.actions + n : nullptr;
         const unsigned long long t_end = a.t0 + (unsigned long long)a.T;
-
         for (unsigned long long c0 = a.t0; c0 < t_end; c0 += kChunk) {
             const unsigned long long c1 = c0 + kChunk < t_end ? c0 + kChunk : t_end;
-            const int filled = 1 + ((int)(c1 - c0) - 1) / 8;
-            for (int k = 0; k < filled; ++k) {
-                Env r;
-                reset_env(r, env_id, (uint32_t)(e.episode + 1 + k), a.rk);
-                table[k][tid] = make_float4(r.x, r.xd, r.th, r.thd);
-            }
-            int used = 0;
-            for (unsigned long long g = c0 >> 2; g <= (c1 - 1) >> 2; ++g) {
-                uint32_t w[4] = {0u, 0u, 0u, 0u};
-                if (MODE == 0) philox((uint32_t)g, env_id, (uint32_t)(g >> 32), 3u, a.rk, w);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const unsigned long long tt = g * 4 + j;
-                    if (FULL || (tt >= c0 && tt < c1)) {
-                        int action;
-                        if (MODE == 0) action = (int)(w[j] & 1u);
-                        else if (MODE == 2) { action = *act & 1u; act += stride; }
-                        else action = a.const_action;
-                        advance(e, action);
-                        const bool done = terminated(e);
-                        if (done) {
-                            episodes += 1;
-                            sum_length += e.steps;
-                            e.episode += 1;
-                            e.steps = 0;
-                            if (used < filled) {
-                                const float4 r = table[used][tid];
-                                e.x = r.x; e.xd = r.y; e.th = r.z; e.thd = r.w;
-                                used += 1;
-                            } else {
-                                reset_env(e, env_id, (uint32_t)e.episode, a.rk);
-                            }
-                        }
-                        *obs = make_float4(e.x, e.xd, e.th, e.thd);
-                        *rew = 1.0f;
-                        *dn = done ? 1 : 0;
-                        obs += stride;
-                        rew += stride;
-                        dn += stride;
-                    }
-                }
-            }
+            run_span<MODE, FULL>(e, env_id, c0, c1, &table[0][tid], kBlock, obs, rew, dn, act, stride, episodes,
+                                 sum_length, a);
         }
         a.plane_f[n] = make_float4(e.x, e.xd, e.th, e.thd);
         a.plane_i[n] = make_int2(e.steps, e.episode);
+    }
+    flush_stats(episodes, sum_length, a.stats);
+}
+
+// ---- balanced chains ----------------------------------------------------------------------
+//
+// With every block resident from the start a launch takes as long as the scheduler that holds
+// the most warps; 65,536 envs are 13.84 warps per SM, which 128-thread blocks place as four
+// blocks (four warps on every scheduler) on 68 SMs and three on the rest.  Here one 16-warp
+// block per SM owns a contiguous range of up to 14 chains (32 consecutive envs, a lane each).
+// Warp w sits on scheduler w % 4.  The first 4 * floor(c / 4) chains stay on warps 0..11; when
+// one or two are left over, each alternates between two warps on different schedulers (12 and
+// 14, 13 and 15) every kChainSpan steps, so that all four schedulers carry the same load.  A
+// hand-over is the six state words through shared memory and one named hardware barrier that
+// both warps execute exactly once per hand-over.  Needs t0 and T to be multiples of 4.
+constexpr int kChainMax = 14;
+constexpr int kChainThreads = 512;
+constexpr int kChainSpan = 32;   // steps a leftover chain runs on one warp (a multiple of 4, <= kChunk)
+constexpr int kChainSmemBytes = kTable * kChainMax * 32 * (int)sizeof(float4) + 2 * 6 * 32 * 4;
+
+__device__ __forceinline__ void named_barrier(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" :: "r"(id), "r"(threads) : "memory");
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kChainThreads, 1) k_cartpole_chains(const __grid_constant__ Args a)
+{
+    extern __shared__ __align__(16) uint8_t chain_smem[];
+    float4 *table = reinterpret_cast<float4 *>(chain_smem);                 // [kTable][kChainMax * 32]
+    uint32_t(*hand)[6][32] = reinterpret_cast<uint32_t(*)[6][32]>(table + kTable * kChainMax * 32);
+    constexpr int pitch = kChainMax * 32;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int groups = (a.n + 31) >> 5;
+    const int g_lo = (int)((long long)blockIdx.x * groups / gridDim.x);
+    const int g_hi = (int)((long long)(blockIdx.x + 1) * groups / gridDim.x);
+    const int c = g_hi - g_lo;          // <= kChainMax (launcher)
+    const int fixed = c & ~3, extra = c & 3;
+
+    // this warp's chain, and which spans of the launch it takes: first, first + 2, ...
+    int chain = -1, span = a.T, first = 0, slot = 0;
+    if (warp < fixed) {
+        chain = warp;
+    } else if (warp >= 12) {
+        const int k = warp - 12;
+        if ((extra == 1 || extra == 2) && fixed >= 4 && a.T > kChainSpan) {
+            if ((k & 1) < extra) {
+                slot = k & 1;
+                chain = fixed + slot;
+                span = kChainSpan;
+                first = k >> 1;
+            }
+        } else if (k < extra) {
+            chain = fixed + k;
+        }
+    }
+    if (chain < 0) return;  // whole warps; no block-wide barrier anywhere
+    const int spans = (a.T + span - 1) / span;
+
+    const int n = (g_lo + chain) * 32 + lane;
+    const bool valid = n < a.n;
+    const int nn = valid ? n : a.n - 1;   // lanes past the batch run a copy of the last env, store nothing
+    const uint32_t env_id = a.env_id_base + (uint32_t)nn;
+    const size_t stride = (size_t)a.n;
+    float4 *column = table + chain * 32 + lane;
+    uint32_t(*h)[32] = hand[slot];
+    int episodes = 0, sum_length = 0;
+    Env e;
+
+    for (int j = first; j < spans; j += 2) {
+        const int ta = j * span, tb = min(a.T, ta + span);
+        if (j == 0) {
+            const float4 f = a.plane_f[nn];
+            const int2 i = a.plane_i[nn];
+            e.x = f.x; e.xd = f.y; e.th = f.z; e.thd = f.w;
+            e.steps = i.x; e.episode = i.y;
+        } else {
+            named_barrier(1 + slot * 2 + ((j - 1) & 1), 64);   // the other warp has written the state
+            e.x = __uint_as_float(h[0][lane]); e.xd = __uint_as_float(h[1][lane]);
+            e.th = __uint_as_float(h[2][lane]); e.thd = __uint_as_float(h[3][lane]);
+            e.steps = (int)h[4][lane]; e.episode = (int)h[5][lane];
+        }
+        if (valid) {
+            float4 *obs = a.obs + (size_t)ta * stride + n;
+            float *rew = a.reward + (size_t)ta * stride + n;
+            uint8_t *dn = a.done + (size_t)ta * stride + n;
+            const uint8_t *act = MODE == 2 ? a.actions + (size_t)ta * stride + n : nullptr;
+            for (int c0 = ta; c0 < tb; c0 += kChunk) {
+                const int c1 = min(tb, c0 + kChunk);
+                run_span<MODE, true>(e, env_id, a.t0 + (unsigned long long)c0, a.t0 + (unsigned long long)c1, column,
+                                     pitch, obs, rew, dn, act, stride, episodes, sum_length, a);
+            }
+        }
+        if (j + 1 < spans) {
+            h[0][lane] = __float_as_uint(e.x); h[1][lane] = __float_as_uint(e.xd);
+            h[2][lane] = __float_as_uint(e.th); h[3][lane] = __float_as_uint(e.thd);
+            h[4][lane] = (uint32_t)e.steps; h[5][lane] = (uint32_t)e.episode;
+            named_barrier(1 + slot * 2 + (j & 1), 64);
+        } else if (valid) {
+            a.plane_f[n] = make_float4(e.x, e.xd, e.th, e.thd);
+            a.plane_i[n] = make_int2(e.steps, e.episode);
+        }
     }
     flush_stats(episodes, sum_length, a.stats);
 }
@@ -273,6 +388,8 @@ struct cartpole_env {
     long long *stats = nullptr;
     uint64_t t = 0;
     int64_t launches = 0;
+    int path = 0;      // CARTPOLE_PATH_*
+    int sms = 0;
     cartpole::RoundKeys rk;
     void *stage = nullptr;
     size_t stage_bytes = 0;
@@ -339,15 +456,38 @@ int do_rollout(cartpole_env *h, int T, int mode, const uint8_t *actions, int con
     a.done = done;
     const int grid = (h->n + cartpole::kBlock - 1) / cartpole::kBlock;
     const bool full = h->t % 4 == 0 && T % 4 == 0;
+    // Balanced chains: from 9 chains of 32 envs on the fullest SM up to the 14 its shared memory
+    // holds (37,889 to 66,304 envs on 148 SMs), or when asked for.  Measured against the 128-env
+    // blocks at T = 128: 45,056 envs 34.7 against 36.1 us, 65,536 envs 39.0 against 45.2 us; equal
+    // below 9 chains per SM, where both are bound by the latency of the step chain.
+    const int groups = (h->n + 31) / 32;
+    const int cgrid = groups < h->sms ? groups : h->sms;
+    const int fullest = (groups + cgrid - 1) / cgrid;
+    const bool chains = full && h->path != CARTPOLE_PATH_PLAIN && fullest <= cartpole::kChainMax &&
+                        (h->path == CARTPOLE_PATH_CHAINS || fullest >= 9);
+    if (chains) {
+#define CARTPOLE_CHAINS(M)                                                                                 \
+    do {                                                                                                   \
+        if (cudaFuncSetAttribute(cartpole::k_cartpole_chains<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                 cartpole::kChainSmemBytes) != cudaSuccess)                                \
+            return CARTPOLE_ECUDA;                                                                         \
+        cartpole::k_cartpole_chains<M><<<cgrid, cartpole::kChainThreads, cartpole::kChainSmemBytes, h->stream>>>(a); \
+    } while (0)
+        if (mode == CARTPOLE_ACT_PHILOX) CARTPOLE_CHAINS(0);
+        else if (mode == CARTPOLE_ACT_EXPLICIT) CARTPOLE_CHAINS(2);
+        else CARTPOLE_CHAINS(3);
+#undef CARTPOLE_CHAINS
+    } else {
 #define CARTPOLE_LAUNCH(M)                                                                       \
     do {                                                                                         \
         if (full) cartpole::k_cartpole_rollout<M, true><<<grid, cartpole::kBlock, 0, h->stream>>>(a);  \
         else cartpole::k_cartpole_rollout<M, false><<<grid, cartpole::kBlock, 0, h->stream>>>(a);      \
     } while (0)
-    if (mode == CARTPOLE_ACT_PHILOX) CARTPOLE_LAUNCH(0);
-    else if (mode == CARTPOLE_ACT_EXPLICIT) CARTPOLE_LAUNCH(2);
-    else CARTPOLE_LAUNCH(3);
+        if (mode == CARTPOLE_ACT_PHILOX) CARTPOLE_LAUNCH(0);
+        else if (mode == CARTPOLE_ACT_EXPLICIT) CARTPOLE_LAUNCH(2);
+        else CARTPOLE_LAUNCH(3);
 #undef CARTPOLE_LAUNCH
+    }
     if (cudaGetLastError() != cudaSuccess) return CARTPOLE_ECUDA;
     h->launches += 1;
     h->t += (uint64_t)T;
@@ -368,6 +508,15 @@ int cartpole_create(cartpole_env **out, int n_envs, uint64_t seed, int env_id_ba
     h->n = n_envs;
     h->seed = seed;
     h->env_id_base = env_id_base;
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&h->sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || h->sms < 1) {
+            cudaGetLastError();
+            delete h;
+            return CARTPOLE_ECUDA;
+        }
+    }
     for (int r = 0; r < 10; ++r) {
         h->rk.k[2 * r] = (uint32_t)seed + (uint32_t)r * cartpole::kW0;
         h->rk.k[2 * r + 1] = (uint32_t)(seed >> 32) + (uint32_t)r * cartpole::kW1;
@@ -544,6 +693,14 @@ int cartpole_set_state(cartpole_env *h, const float *host_f, const int32_t *host
         cudaStreamSynchronize(h->stream) != cudaSuccess)
         return CARTPOLE_ECUDA;
     h->t = t;
+    return CARTPOLE_OK;
+}
+
+int cartpole_set_path(cartpole_env *h, int path)
+{
+    if (h == nullptr) return CARTPOLE_ENULL;
+    if (path < CARTPOLE_PATH_AUTO || path > CARTPOLE_PATH_CHAINS) return CARTPOLE_EINVAL;
+    h->path = path;
     return CARTPOLE_OK;
 }
 

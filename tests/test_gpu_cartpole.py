@@ -222,3 +222,38 @@ def test_full_size_sampled(torch):
         assert bool((reward == 1.0).all()) and bool((done <= 1).all())
     ep, length = env.episode_stats()
     assert ep == total_done > n and 15 < length / ep < 30
+
+
+@pytest.mark.parametrize("n,T,mode", [
+    (1, 4, 0), (40, 64, 0), (1000, 128, 2), (4097, 36, 3),
+    (26048, 100, 0), (26033, 64, 2), (33152, 68, 0), (45056, 128, 0),
+    (61568, 32, 0), (65536, 128, 0), (65536, 36, 2), (66304, 160, 3), (66290, 96, 0),
+])
+def test_chains_path_matches_the_oracle(torch, n, T, mode):
+    """The balanced-chains kernel with the path forced, element by element: one chain per block,
+    4 + 1 / 4 + 2 chains (leftovers alternating between two warps every 32 steps), 4 + 3 (whole
+    leftovers), 8 + 1 / 8 + 2, 12 + 1 / 12 + 2, the largest batch, ragged last chains; rollouts of
+    one span, whole spans and a short last span.  CartPole episodes end every ~22 steps, so every
+    span crosses resets."""
+    seed = 300 + n % 89
+    env, ora = cp.CartPoleEnv(n, seed, env_id_base=11), ocp.OracleCartPole(n, seed, env_id_base=11)
+    env.set_path(cp.PATH_CHAINS)
+    for rep in range(2):
+        if mode == 2:
+            a = actions(T, n, rep)
+            g, o = env.rollout(T, 2, torch.from_numpy(a).cuda()), ora.rollout(T, 2, a)
+        elif mode == 3:
+            g, o = env.rollout(T, 3, rep), ora.rollout(T, 3, rep)
+        else:
+            g, o = env.rollout(T, 0), ora.rollout(T, 0)
+        assert_equal(g, o, "chains n %d T %d mode %d launch %d" % (n, T, mode, rep))
+    # an unaligned call falls back to the plain kernel, and the chains kernel picks up again after it
+    g, o = env.rollout(3, 0), ora.rollout(3, 0)
+    assert_equal(g, o, "unaligned")
+    g, o = env.rollout(1, 0), ora.rollout(1, 0)
+    assert_equal(g, o, "realign")
+    g, o = env.rollout(64, 0), ora.rollout(64, 0)
+    assert_equal(g, o, "chains again")
+    assert_state_equal(env, ora)
+    with pytest.raises(cp.CartPoleError):
+        env.set_path(5)
