@@ -74,11 +74,11 @@ WORKLOADS = {
     "cartpole65k": dict(
         name="CartPole fused rollout, N=65536 envs, T=128 steps per launch, in-kernel Philox actions",
         env="cartpole", n=65536, T=128, mode=0, obs_mode=0, frameskip=1, bytes=21.0 + 48.0 / 128,
-        kernel="k_cartpole_chains", traffic=None),
+        kernel="k_cartpole_chains", traffic=176.07e6),
     "cartpole1m": dict(
         name="CartPole fused rollout, N=1048576 envs, T=32 steps per launch, in-kernel Philox actions",
         env="cartpole", n=1048576, T=32, mode=0, obs_mode=0, frameskip=1, bytes=21.0 + 48.0 / 32,
-        kernel="k_cartpole_rollout", traffic=None),
+        kernel="k_cartpole_rollout", traffic=753.6e6),
     "policy65k": dict(
         name="policy in the loop: gru_policy_encode -> gru_policy_cell (tcgen05, 2.0 M parameters, bf16) -> "
              "gru_policy_head -> pong_sample_actions -> pong_step, N=65536 envs, 32 agent steps per "
