@@ -13,9 +13,10 @@ statistics reduction, i.e. 8,388,608 env-steps and 243 MB written per step.
                                 cartpole65k|cartpole1m|policy65k]
 
 Timing follows the paper's protocol (warm-up excluded, mean and spread over at least
-five runs): a block of K launches (--steps) is repeated, back to back, until at least
-0.25 s of device time and five repeats are in the timed region; `value` comes from the
-whole region, `segments` holds the per-repeat rates, clocks are sampled inside it.
+five runs): five repeats are timed, each made of as many whole blocks of K launches
+(--steps) as it takes to put at least 0.25 s of device time into the timed region, all
+back to back with CUDA events between repeats only; `value` comes from the whole region,
+`segments` holds the per-repeat rates, clocks are sampled inside it.
 The default run also appends one short record for each of the other configurations
 ("configs").
 
@@ -304,25 +305,25 @@ def run_policy(args, w, rank, world, local, full=True):
         for _ in range(warmup):
             loop.replay()
         loop.sync_and_check()
-        per_ms, ms_total, w0, w1 = timed_blocks(loop.replay, steps, barrier, max_ranks,
-                                                min_seconds=args.min_seconds)
+        per_ms, ms_total, w0, w1, blocks = timed_blocks(loop.replay, steps, barrier, max_ranks,
+                                                        min_seconds=args.min_seconds)
         loop.sync_and_check()
         # launches made while capturing are replayed: count kernels per replay from what a step launches
         per_replay = parts * (K * ((3 if with_policy else 0) + (2 if with_env else 0)) + (1 if with_env else 0))
-        return per_ms, max_ranks(ms_total), w0, w1, loop, len(per_ms) * steps * per_replay
+        return per_ms, max_ranks(ms_total), w0, w1, loop, len(per_ms) * blocks * steps * per_replay, blocks
 
     sampler = ClockSampler(physical_gpu_index(local))
     sampler.start()
-    per_ms, ms_env, w0, w1, loop, launches = timed(True)
+    per_ms, ms_env, w0, w1, loop, launches, blocks = timed(True)
     repeats = len(per_ms)
-    replays = repeats * steps
+    replays = repeats * blocks * steps
     clocks = sampler.summary(w0, w1)
     ms_pol = ms_envk = None
     if full:
-        p2, ms_pol, _, _, _, _ = timed(False)
-        ms_pol /= len(p2) * steps
-        p3, ms_envk, _, _, _, _ = timed(True, with_policy=False)
-        ms_envk /= len(p3) * steps
+        p2, ms_pol, _, _, _, _, b2 = timed(False)
+        ms_pol /= len(p2) * b2 * steps
+        p3, ms_envk, _, _, _, _, b3 = timed(True, with_policy=False)
+        ms_envk /= len(p3) * b3 * steps
     # the cell kernel alone, back to back, all N envs per launch, on operands of the loop's kind
     policy._stream()
     gen = torch.Generator(device="cuda:%d" % local).manual_seed(SEED)
@@ -357,7 +358,7 @@ def run_policy(args, w, rank, world, local, full=True):
     sampler.stop()
     ms_replay = ms_env / replays
     value = world * N * K / (ms_replay * 1e-3)
-    seg = spread([steps * N * K / (m * 1e-3) for m in per_ms])
+    seg = spread([blocks * steps * N * K / (m * 1e-3) for m in per_ms])
     cell_flops = 2.0 * 6 * hidden * hidden * N          # the six H x H products of one agent step
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
@@ -378,13 +379,13 @@ def run_policy(args, w, rank, world, local, full=True):
         return {"workload_key": "policy65k", "workload": w["name"], "value": value, "unit": UNIT,
                 "us_per_launch": ms_replay * 1e3, "agent_step_us": ms_replay / K * 1e3,
                 "cell_kernel_us": cell_ms * 1e3, "steps": steps, "repeats": repeats,
-                "roofline": roofline, "segments": seg, "clocks": clocks,
+                "blocks_per_repeat": blocks, "roofline": roofline, "segments": seg, "clocks": clocks,
                 "dtype": "bf16 policy (f32 accumulate), int32 env", "gpu_launches": int(launches)}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": ms_replay, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16 policy (f32 accumulate), int32 env", "data": "synthetic",
-        "repeats": repeats,
+        "repeats": repeats, "blocks_per_repeat": blocks,
         "config": {"workload": w["name"], "workload_key": args.workload, "n_envs_per_gpu": N,
                    "agent_steps_per_graph": K, "policy_parameters": n_params, "hidden": hidden,
                    "parallel_slices": parts,
@@ -418,12 +419,14 @@ def run_policy(args, w, rank, world, local, full=True):
     return line
 
 
-def timed_blocks(launch, steps, barrier, max_over_ranks, min_seconds=0.25, min_repeats=5, max_repeats=4000):
+def timed_blocks(launch, steps, barrier, max_over_ranks, min_seconds=0.25, min_repeats=5):
     """Times blocks of `steps` launches, back to back, with CUDA events on the launching
-    stream: one untimed block sizes the run, then the block is repeated until the timed
-    work is at least min_seconds and there are at least min_repeats repeats (the paper's
-    protocol: warm-up excluded, mean and spread over N >= 5 runs).  Returns the per-repeat
-    times in ms, the total in ms, and the wall-clock bracket of the timed region."""
+    stream: one untimed block sizes the run, then min_repeats repeats are timed, each made
+    of as many whole blocks as it takes for the repeats to add up to min_seconds of device
+    time (the paper's protocol: warm-up excluded, mean and spread over N >= 5 runs).  Events
+    sit between repeats only, so the launches inside a repeat run back to back whatever
+    `steps` is.  Returns the per-repeat times in ms, the total in ms, the wall-clock bracket
+    of the timed region and the number of blocks per repeat."""
     import torch
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
@@ -431,21 +434,21 @@ def timed_blocks(launch, steps, barrier, max_over_ranks, min_seconds=0.25, min_r
         launch()
     e1.record()
     torch.cuda.synchronize()
-    probe_ms = max_over_ranks(e0.elapsed_time(e1))
-    repeats = int(min(max_repeats, max(min_repeats, -(-min_seconds * 1e3 // max(probe_ms, 1e-3)))))
+    probe_ms = max(max_over_ranks(e0.elapsed_time(e1)), 1e-3)
+    blocks = int(max(1, -(-(min_seconds * 1e3 / min_repeats) // probe_ms)))
     barrier()
-    marks = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 1)]
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(min_repeats + 1)]
     w0 = time.perf_counter()
     marks[0].record()
-    for r in range(repeats):
-        for _ in range(steps):
+    for r in range(min_repeats):
+        for _ in range(blocks * steps):
             launch()
         marks[r + 1].record()
     torch.cuda.synchronize()
     w1 = time.perf_counter()
     barrier()
-    per = [marks[r].elapsed_time(marks[r + 1]) for r in range(repeats)]
-    return per, marks[0].elapsed_time(marks[-1]), w0, w1
+    per = [marks[r].elapsed_time(marks[r + 1]) for r in range(min_repeats)]
+    return per, marks[0].elapsed_time(marks[-1]), w0, w1, blocks
 
 
 def spread(values):
@@ -530,12 +533,12 @@ def run_env(args, key, rank, world, local, full):
 
     # ---- device-resident timing: repeated blocks of `steps` launches, CUDA events on the launching stream
     launches0 = env.launches
-    per_ms, ms_total, w0, w1 = timed_blocks(launch, steps, barrier, max_ranks,
-                                            min_seconds=args.min_seconds)
+    per_ms, ms_total, w0, w1, blocks = timed_blocks(launch, steps, barrier, max_ranks,
+                                                    min_seconds=args.min_seconds)
     launches = env.launches - launches0 - steps        # without the untimed sizing block
     repeats = len(per_ms)
     ms_total = max_ranks(ms_total)
-    seg = spread([steps * env_steps_per_launch / (m * 1e-3) for m in per_ms])
+    seg = spread([blocks * steps * env_steps_per_launch / (m * 1e-3) for m in per_ms])
     clocks = sampler.summary(w0, w1)
     stats = sharding.sum_stats(env.episode_stats(), device="cuda")
 
@@ -597,7 +600,7 @@ def run_env(args, key, rank, world, local, full):
     sampler.stop()
     barrier()
 
-    total_launches = repeats * steps
+    total_launches = repeats * blocks * steps
     value = world * total_launches * env_steps_per_launch / (ms_total * 1e-3)
     peak, peak_kind = measured_peak()
     kernel_ms = ms_total / total_launches
@@ -630,7 +633,7 @@ def run_env(args, key, rank, world, local, full):
     if not full:
         rec = {"workload_key": key, "workload": w["name"], "value": value, "unit": UNIT,
                "us_per_launch": kernel_ms * 1e3, "steps": steps, "repeats": repeats,
-               "bytes_per_env_step": w["bytes"], "achieved_gbs": achieved,
+               "blocks_per_repeat": blocks, "bytes_per_env_step": w["bytes"], "achieved_gbs": achieved,
                "frac_of_measured": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
                "kernel": w["kernel"], "segments": seg, "clocks": clocks,
                "dtype": "f32" if is_cartpole else "int32", "gpu_launches": int(launches)}
@@ -643,14 +646,14 @@ def run_env(args, key, rank, world, local, full):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": kernel_ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32" if is_cartpole else "int32",
-        "data": "synthetic", "repeats": repeats,
+        "data": "synthetic", "repeats": repeats, "blocks_per_repeat": blocks,
         "config": {
             "workload": w["name"], "workload_key": key, "n_envs_per_gpu": N, "T": T,
             "frameskip": w["frameskip"], "seed": SEED, "env_steps_per_step": env_steps_per_launch,
             "l2": l2_note,
-            "timing": "%d repeats of a block of %d launches, back to back, CUDA events between "
-                      "blocks; value from the whole timed region, segments = per-repeat rates"
-                      % (repeats, steps),
+            "timing": "%d repeats of %d blocks of %d launches each, back to back, CUDA events between "
+                      "repeats; value from the whole timed region, segments = per-repeat rates"
+                      % (repeats, blocks, steps),
             "parallelism": "env shards per GPU, no collective" if world > 1 else "single GPU",
         },
         "roofline": roofline,
@@ -669,8 +672,8 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=0,
-                    help="launches per timed block (default: per workload); blocks repeat until "
-                         "--min-seconds of timed work and at least 5 repeats")
+                    help="launches per block (default: per workload); five repeats of as many blocks "
+                         "as it takes to time --min-seconds of work")
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--workload", default="rollout65k", choices=sorted(WORKLOADS))

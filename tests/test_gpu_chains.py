@@ -44,6 +44,7 @@ def run_pair(env, ora, T, mode, seed):
     (16, 8, 0), (48, 16, 1), (1040, 24, 2), (4112, 40, 3),
     (26048, 24, 0), (26048, 40, 1), (26048, 72, 0), (33152, 24, 0), (45056, 40, 2), (45056, 64, 1),
     (61568, 16, 0), (65536, 40, 0), (65536, 72, 1), (65536, 48, 2), (66304, 64, 3), (66288, 128, 0),
+    (65536, 128, 0),
 ])
 def test_chains_path_matches_the_oracle(torch_cuda, n, T, mode):
     seed, base = 1000 + n % 97, 3
