@@ -137,6 +137,10 @@ __global__ void __launch_bounds__(kVecBlock) k_rollout_vector(const __grid_const
     const int n = blockIdx.x * kVecBlock + threadIdx.x;
     const bool valid = n < a.n;
     Tally tally = {0, 0, 0};
+    // launched with the programmatic-dependent-launch attribute: the block may be resident before
+    // the preceding kernel of the stream (the previous step, or whatever produced the actions) has
+    // finished; nothing of the caller's or the handle's memory is touched before this wait
+    grid_dependency_wait();
     if (valid) {
         Env e;
         load_env(e, a.plane0, a.plane1, n);
@@ -170,6 +174,7 @@ __global__ void __launch_bounds__(kVecBlock) k_rollout_vector(const __grid_const
                 }
             }
         }
+        grid_dependency_launch();
         store_env(e, a.plane0, a.plane1, n);
     }
     flush_tally(tally, a.stats);
@@ -178,11 +183,19 @@ __global__ void __launch_bounds__(kVecBlock) k_rollout_vector(const __grid_const
 template <int MODE, int FS>
 static void launch_vec_full(const LaunchArgs &a, bool full, cudaStream_t s)
 {
-    const int grid = (a.n + kVecBlock - 1) / kVecBlock;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((a.n + kVecBlock - 1) / kVecBlock);
+    cfg.blockDim = dim3(kVecBlock);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (full)
-        k_rollout_vector<MODE, FS, true><<<grid, kVecBlock, 0, s>>>(a);
+        cudaLaunchKernelEx(&cfg, k_rollout_vector<MODE, FS, true>, a);
     else
-        k_rollout_vector<MODE, FS, false><<<grid, kVecBlock, 0, s>>>(a);
+        cudaLaunchKernelEx(&cfg, k_rollout_vector<MODE, FS, false>, a);
 }
 
 template <int MODE>
