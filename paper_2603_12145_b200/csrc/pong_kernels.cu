@@ -272,6 +272,16 @@ __global__ void __launch_bounds__(kTmaBlock) k_rollout_vector_tma(const __grid_c
         // the store that last read this buffer is the older of the two in flight
         if (tid == 0) bulk_wait_read<1>();
         __syncthreads();
+        // reward and done rows start as zeros; a lane writes its entry only on a point or an
+        // episode end (5 x 16-byte stores per thread-pair instead of two stores per step)
+        {
+            uint4 *zr = reinterpret_cast<uint4 *>(&s_reward[buf][0][0]);   // 8 x 64 floats = 128 uint4
+            zr[tid] = make_uint4(0u, 0u, 0u, 0u);
+            zr[tid + kTmaBlock] = make_uint4(0u, 0u, 0u, 0u);
+            uint4 *zd = reinterpret_cast<uint4 *>(&s_done[buf][0][0]);     // 8 x 64 bytes = 32 uint4
+            if (tid < kTmaStage * kTmaBlock / 16) zd[tid] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        __syncthreads();
 #pragma unroll
         for (int q = 0; q < kTmaStage / 4; ++q) {
             const uint32_t w[4] = {pipe.c0, pipe.c1, pipe.c2, pipe.c3};
@@ -294,15 +304,11 @@ __global__ void __launch_bounds__(kTmaBlock) k_rollout_vector_tma(const __grid_c
                 else if (MODE == 2) action = decode_action_byte(abyte[s], e.prev);
                 else action = a.const_action;
                 e.prev = action;
-                float r;
-                int dn;
-                fast_frame<QUEUE>(e, action, env_id, a.rk, tally, r, dn);
+                fast_frame<QUEUE>(e, action, env_id, a.rk, tally, &s_reward[buf][s][tid], &s_done[buf][s][tid]);
                 float2 *o = reinterpret_cast<float2 *>(&s_obs[buf][s][tid * 6]);
                 o[0] = make_float2(scale_obs(e.bx), scale_obs(e.by));
                 o[1] = make_float2(scale_obs(e.vx), scale_obs(e.vy));
                 o[2] = make_float2(scale_obs(e.apy), scale_obs(e.opy));
-                s_reward[buf][s][tid] = r;
-                s_done[buf][s][tid] = (uint8_t)dn;
             }
         }
         fence_async_smem();
@@ -582,6 +588,15 @@ k_rollout_vector_chains(const __grid_constant__ LaunchArgs a, const __grid_const
             // this warp's own store that last read the buffer is the older of its two in flight
             if (lane == 0) bulk_wait_read<1>();
             __syncwarp();
+            // reward and done rows start as zeros; a lane writes its entry only on a point or an
+            // episode end
+            {
+                uint4 *zr = reinterpret_cast<uint4 *>(&st.reward[0][0]);   // 8 x 32 floats = 64 uint4
+                zr[lane] = make_uint4(0u, 0u, 0u, 0u);
+                zr[lane + 32] = make_uint4(0u, 0u, 0u, 0u);
+                if (lane < kTmaStage * 32 / 16) reinterpret_cast<uint4 *>(&st.done[0][0])[lane] = make_uint4(0u, 0u, 0u, 0u);
+            }
+            __syncwarp();
 #pragma unroll
             for (int q = 0; q < kTmaStage / 4; ++q) {
                 const uint32_t w[4] = {pipe.c0, pipe.c1, pipe.c2, pipe.c3};
@@ -604,15 +619,11 @@ k_rollout_vector_chains(const __grid_constant__ LaunchArgs a, const __grid_const
                     else if (MODE == 2) action = decode_action_byte(abyte[k], e.prev);
                     else action = a.const_action;
                     e.prev = action;
-                    float r;
-                    int dn;
-                    fast_frame<QUEUE>(e, action, env_id, a.rk, tally, r, dn);
+                    fast_frame<QUEUE>(e, action, env_id, a.rk, tally, &st.reward[k][lane], &st.done[k][lane]);
                     float2 *o = reinterpret_cast<float2 *>(&st.obs[k][lane * 6]);
                     o[0] = make_float2(scale_obs(e.bx), scale_obs(e.by));
                     o[1] = make_float2(scale_obs(e.vx), scale_obs(e.vy));
                     o[2] = make_float2(scale_obs(e.apy), scale_obs(e.opy));
-                    st.reward[k][lane] = r;
-                    st.done[k][lane] = (uint8_t)dn;
                 }
             }
             fence_async_smem();

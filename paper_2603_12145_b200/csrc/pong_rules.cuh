@@ -282,10 +282,12 @@ __device__ __forceinline__ uint32_t spawn_entry(uint32_t env_id, uint32_t episod
 
 // Score and / or episode end.  Run by the whole warp when any lane has an event;
 // only lanes with `ev` commit.  `out` says the ball left the court on this lane.
+// `reward` and `done` point at this lane's entries of the staged output rows, which the caller
+// has zeroed: only a lane with an event writes them.
 template <bool QUEUE>
 __device__ __forceinline__ void fast_event(FastEnv &e, bool ev, bool out, uint32_t env_id,
-                                           const RoundKeys &rk, Tally &tally, float &reward,
-                                           int &done)
+                                           const RoundKeys &rk, Tally &tally, float *reward,
+                                           uint8_t *done)
 {
     const bool agent_point = e.bx > 0;
     int sa = e.sa + ((out && agent_point) ? 1 : 0);
@@ -323,17 +325,18 @@ __device__ __forceinline__ void fast_event(FastEnv &e, bool ev, bool out, uint32
         e.bx = kSpawnBx; e.by = kSpawnBy;
         e.vx = (ent & 0x400u) ? kVx0 : -kVx0;
         e.vy = (int)(ent & 0x3FFu) - kVySpawn;
-        reward = r;
-        done = dn ? 1 : 0;
+        *reward = r;
+        *done = dn ? 1 : 0;
         if (dn) { e.left = kMaxFrames; e.apy = kPadY0; e.opy = kPadY0; e.prev = 0; }
     }
 }
 
-// One frame; all 32 lanes of the warp must call it together.
+// One frame; all 32 lanes of the warp must call it together.  The reward and done entries
+// (pre-zeroed by the caller) are written only on a point or an episode end.
 template <bool QUEUE>
 __device__ __forceinline__ void fast_frame(FastEnv &e, int action, uint32_t env_id,
-                                           const RoundKeys &rk, Tally &tally, float &reward,
-                                           int &done)
+                                           const RoundKeys &rk, Tally &tally, float *reward,
+                                           uint8_t *done)
 {
     const int delta = action == 2 ? kAgentStep : (action == 1 ? -kAgentStep : 0);
     e.apy = min(max(e.apy + delta, 0), kPadYMax);
@@ -361,8 +364,6 @@ __device__ __forceinline__ void fast_frame(FastEnv &e, int action, uint32_t env_
     e.left -= 1;
     const bool out = (unsigned)e.bx > (unsigned)kCourtW;
     const bool ev = out || e.left == 0;
-    reward = 0.f;
-    done = 0;
     if (__any_sync(0xffffffffu, ev)) fast_event<QUEUE>(e, ev, out, env_id, rk, tally, reward, done);
 }
 
