@@ -113,9 +113,11 @@ __device__ __forceinline__ void action_words(uint64_t group, uint32_t env_id,
     philox4x32_10((uint32_t)group, env_id, (uint32_t)(group >> 32), 0u, rk, w);
 }
 
+// (u * 3) >> 16 for the low half-word u, written as the high word of (u << 16) * 3: a shift
+// and a multiply-high (which runs on the multiply pipe, not the integer ALU's).
 __device__ __forceinline__ int uniform_action(uint32_t word)
 {
-    return (int)(((word & 0xFFFFu) * 3u) >> 16);
+    return (int)__umulhi(word << 16, 3u);
 }
 
 __device__ __forceinline__ bool sticky_repeat(uint32_t word)
@@ -338,7 +340,9 @@ __device__ __forceinline__ void fast_frame(FastEnv &e, int action, uint32_t env_
                                            const RoundKeys &rk, Tally &tally, float *reward,
                                            uint8_t *done)
 {
-    const int delta = action == 2 ? kAgentStep : (action == 1 ? -kAgentStep : 0);
+    // 0, -768, +768 for action 0, 1, 2 as the polynomial (1152 a - 1920) a: two multiply-adds
+    // on the multiply pipe instead of two compares and two selects on the integer ALU
+    const int delta = (action * (3 * kAgentStep / 2) - (5 * kAgentStep / 2)) * action;
     e.apy = min(max(e.apy + delta, 0), kPadYMax);
     const int d = e.by - e.opy - 1792;
     e.opy = min(max(e.opy + min(max(d, -kOppStep), kOppStep), 0), kPadYMax);
