@@ -35,7 +35,9 @@
  * DEVICE pointer owned by the caller unless its name says host; step / rollout
  * / reset enqueue on the handle's stream and return; episode_stats / get_state
  * / set_state synchronise it.  Return 0 or a negative CARTPOLE_E* code; no
- * exceptions, aborts, traps or printing; no CPU fallback.
+ * exceptions, aborts, traps or printing; no CPU fallback.  A handle is not
+ * thread-safe, and the library fills a small per-device cache on first use
+ * without a lock: make the first rollout on each device from one thread.
  */
 #ifndef CARTPOLE_H_
 #define CARTPOLE_H_

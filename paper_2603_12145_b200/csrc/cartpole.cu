@@ -466,11 +466,19 @@ int do_rollout(cartpole_env *h, int T, int mode, const uint8_t *actions, int con
     const bool chains = full && h->path != CARTPOLE_PATH_PLAIN && fullest <= cartpole::kChainMax &&
                         (h->path == CARTPOLE_PATH_CHAINS || fullest >= 9);
     if (chains) {
+        // the kernel's shared-memory limit is raised once per device and action mode (an unlocked
+        // cache: a second thread at worst sets the same value again)
+        static bool limit_set[4][64] = {};
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) dev = 0;
 #define CARTPOLE_CHAINS(M)                                                                                 \
     do {                                                                                                   \
-        if (cudaFuncSetAttribute(cartpole::k_cartpole_chains<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                                 cartpole::kChainSmemBytes) != cudaSuccess)                                \
-            return CARTPOLE_ECUDA;                                                                         \
+        if (!limit_set[M][dev]) {                                                                          \
+            if (cudaFuncSetAttribute(cartpole::k_cartpole_chains<M>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                     cartpole::kChainSmemBytes) != cudaSuccess)                            \
+                return CARTPOLE_ECUDA;                                                                     \
+            limit_set[M][dev] = true;                                                                      \
+        }                                                                                                  \
         cartpole::k_cartpole_chains<M><<<cgrid, cartpole::kChainThreads, cartpole::kChainSmemBytes, h->stream>>>(a); \
     } while (0)
         if (mode == CARTPOLE_ACT_PHILOX) CARTPOLE_CHAINS(0);
