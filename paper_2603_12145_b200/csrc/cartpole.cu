@@ -142,8 +142,10 @@ __device__ __forceinline__ void advance(Env &e, int action)
 
 __device__ __forceinline__ bool terminated(const Env &e)
 {
+    // x < -L || x > L is |x| > L (false for a NaN either way); the absolute value is an operand
+    // modifier of the compare, not an instruction
     const float th_limit = 0.20943951023931953f;
-    return e.x < -2.4f || e.x > 2.4f || e.th < -th_limit || e.th > th_limit || e.steps >= kMaxSteps;
+    return fabsf(e.x) > 2.4f || fabsf(e.th) > th_limit || e.steps >= kMaxSteps;
 }
 
 __device__ __forceinline__ void flush_stats(int episodes, int sum_length, long long *stats)
