@@ -59,11 +59,11 @@ WORKLOADS = {
     "rollout65k": dict(
         name="fused vector-obs rollout, N=65536 envs, T=128 steps per launch, in-kernel Philox actions",
         n=65536, T=128, mode=0, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 128,
-        kernel="k_rollout_vector_chains", traffic=244.07e6, alu_per_warp_step=55.5),
+        kernel="k_rollout_vector_chains", traffic=243.7e6, alu_per_warp_step=48.1),
     "rollout1m": dict(
         name="fused vector-obs rollout, N=1048576 envs, T=32 steps per launch, in-kernel Philox sticky actions",
         n=1048576, T=32, mode=1, obs_mode=0, frameskip=1, bytes=29.0 + 64.0 / 32,
-        kernel="k_rollout_vector_tma", traffic=1038.9e6, alu_per_warp_step=44.5),
+        kernel="k_rollout_vector_tma", traffic=1038.8e6, alu_per_warp_step=38.9),
     "pixels16k": dict(
         name="pixel-obs rollout, N=16384 envs, T=64 agent steps per launch, frameskip 4, 4-frame ring uint8[N,4,84,84]",
         n=16384, T=64, mode=0, obs_mode=1, frameskip=4, bytes=7056.0 + 5.0 + 64.0 / 64,
@@ -75,7 +75,7 @@ WORKLOADS = {
     "cartpole65k": dict(
         name="CartPole fused rollout, N=65536 envs, T=128 steps per launch, in-kernel Philox actions",
         env="cartpole", n=65536, T=128, mode=0, obs_mode=0, frameskip=1, bytes=21.0 + 48.0 / 128,
-        kernel="k_cartpole_chains", traffic=176.07e6),
+        kernel="k_cartpole_chains", traffic=176.4e6),
     "cartpole1m": dict(
         name="CartPole fused rollout, N=1048576 envs, T=32 steps per launch, in-kernel Philox actions",
         env="cartpole", n=1048576, T=32, mode=0, obs_mode=0, frameskip=1, bytes=21.0 + 48.0 / 32,
