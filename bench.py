@@ -67,7 +67,7 @@ WORKLOADS = {
     "pixels16k": dict(
         name="pixel-obs rollout, N=16384 envs, T=64 agent steps per launch, frameskip 4, 4-frame ring uint8[N,4,84,84]",
         n=16384, T=64, mode=0, obs_mode=1, frameskip=4, bytes=7056.0 + 5.0 + 64.0 / 64,
-        kernel="k_rollout_pixels_x4", traffic=7215.5e6),
+        kernel="k_rollout_pixels_x4", traffic=7271.0e6),
     "step4096": dict(
         name="single-step API pong_step, N=4096 envs, one agent step per launch, actions from a device buffer",
         n=4096, T=1, mode=2, obs_mode=0, frameskip=1, bytes=94.0,
