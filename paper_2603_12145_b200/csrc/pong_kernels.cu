@@ -482,6 +482,10 @@ constexpr int kChainWarps = 16;
 constexpr int kChainThreads = kChainWarps * 32;
 constexpr int kChainSegment = 4;              // stages a leftover chain runs on one warp (1: 43.8 us, 2: 41.7, 3: 41.4, 4: 40.9, 5: 41.3, 8: 42.9 at 65,536 x 128)
 constexpr int kHandWords = 12;                // FastEnv as 32-bit words
+// stages between two block-wide rendezvous of the chains (T = 128 / 256 / 512 / 1024 at 65,536 envs:
+// none 40.6 / 82.2 / 172.9 / 359.4 us, every 4: 45.1 / 85.7 / 167.0 / 328.4, every 8: 41.3 / 78.3 /
+// 151.8 / 299.5, every 16: 40.5 / 76.9 / 150.5 / 305.0, every 32: 40.7 / 80.9 / 163.3 / 327.3)
+constexpr int kChainLockstep = 16;
 
 struct ChainStage {
     float obs[kTmaStage][32 * 6];
@@ -585,6 +589,12 @@ k_rollout_vector_chains(const __grid_constant__ LaunchArgs a, const __grid_const
                 peer_buffer_pending = false;
             }
             ChainStage &st = mine[s & 1];
+            // Every kChainLockstep stages the block's chains wait for one another.  Left alone they
+            // drift apart (a chain never waits for another), and once neighbouring chains write
+            // time rows that are far apart the DRAM pages of a row are no longer filled in one go:
+            // a 1024-step launch ran at 5.4 TB/s without this and runs at 6.4 TB/s with it.  Each
+            // chain has exactly one owner warp at any stage, so 32 * c threads arrive per phase.
+            if ((s & (kChainLockstep - 1)) == 0) named_barrier(9, 32 * c);
             // this warp's own store that last read the buffer is the older of its two in flight
             if (lane == 0) bulk_wait_read<1>();
             __syncwarp();

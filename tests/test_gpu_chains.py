@@ -4,7 +4,7 @@ the C ABI with the path forced.  Sizes are chosen so that blocks on a 148-SM par
 every mix the kernel distinguishes: one chain, 4 + 1 / 4 + 2 (alternating leftovers),
 4 + 3 (whole leftovers), 8 + 1 / 8 + 2, 12 + 1 / 12 + 2, the largest batch the kernel
 takes, a ragged last chain; stage counts 1, 2, 3 (no alternation), 5 and 9 (a last segment of one
-stage), 6, 8, 16."""
+stage), 6, 8, 16, and 17, 33, 49 (launches long enough for the block-wide rendezvous every 16 stages)."""
 import numpy as np
 import pytest
 
@@ -44,7 +44,7 @@ def run_pair(env, ora, T, mode, seed):
     (16, 8, 0), (48, 16, 1), (1040, 24, 2), (4112, 40, 3),
     (26048, 24, 0), (26048, 40, 1), (26048, 72, 0), (33152, 24, 0), (45056, 40, 2), (45056, 64, 1),
     (61568, 16, 0), (65536, 40, 0), (65536, 72, 1), (65536, 48, 2), (66304, 64, 3), (66288, 128, 0),
-    (65536, 128, 0),
+    (65536, 128, 0), (65536, 264, 0), (26048, 136, 1), (45056, 392, 0),
 ])
 def test_chains_path_matches_the_oracle(torch_cuda, n, T, mode):
     seed, base = 1000 + n % 97, 3
