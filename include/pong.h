@@ -138,7 +138,9 @@ int pong_set_stream(pong_env *h, void *cuda_stream);
  * blocks, shared-memory staging, TMA tensor stores.  CHAINS: one block per SM,
  * warp chains balanced over the SM's schedulers.  A forced path the call does
  * not qualify for (alignment, T % 8, frameskip, more than 14 x 32 envs per SM)
- * falls through chains -> tma -> general. */
+ * falls through chains -> tma -> general.  Unless the path is GENERAL, a call whose first
+ * step is no multiple of 4 or whose length is no multiple of 8 is run as up to three kernels
+ * (general head, fast middle, general tail) when the middle is at least 16 steps. */
 #define PONG_PATH_AUTO    0
 #define PONG_PATH_GENERAL 1
 #define PONG_PATH_TMA     2

@@ -77,15 +77,16 @@ int do_rollout(pong_env *h, int T, int action_mode, const uint8_t *actions, int 
     a.reward = reward;
     a.done = done;
     cudaError_t err;
+    int kernels = 1;
     if (h->cfg.obs_mode == PONG_OBS_VECTOR) {
         a.obs = static_cast<float *>(obs);
-        err = pong::launch_rollout_vector(a, h->stream, &h->map_cache);
+        err = pong::launch_rollout_vector(a, h->stream, &h->map_cache, &kernels);
     } else {
         a.ring = static_cast<uint8_t *>(obs);
         err = pong::launch_rollout_pixels(a, h->sm_count, h->stream);
     }
     if (err != cudaSuccess) return PONG_ECUDA;
-    h->launches += 1;
+    h->launches += kernels;
     h->t += (uint64_t)T;
     return PONG_OK;
 }

@@ -733,7 +733,8 @@ static bool try_launch_vector_chains(const LaunchArgs &a, cudaStream_t s, cudaEr
     return true;
 }
 
-cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s, VectorMapCache *cache)
+// One kernel for the whole call: a fast kernel if the call qualifies, else the general one.
+static cudaError_t launch_vector_one(const LaunchArgs &a, cudaStream_t s, VectorMapCache *cache)
 {
     cudaError_t fast_err = cudaSuccess;
     if ((a.vector_path == kPathAuto || a.vector_path == kPathChains) &&
@@ -749,6 +750,58 @@ cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s, VectorMap
     default: launch_vec_mode<3>(a, full, s); break;
     }
     return cudaGetLastError();
+}
+
+// The steps [from, from + count) of the call `a` as a call of their own.
+static LaunchArgs sub_call(const LaunchArgs &a, int from, int count)
+{
+    LaunchArgs b = a;
+    const size_t rows = (size_t)from * (size_t)a.n;
+    b.t0 = a.t0 + (unsigned long long)from;
+    b.T = count;
+    b.obs = a.obs + rows * 6;
+    b.reward = a.reward + rows;
+    b.done = a.done + rows;
+    if (a.actions != nullptr && a.action_mode == 2) b.actions = a.actions + rows;
+    return b;
+}
+
+// A call that misses the fast kernels only because its first step is not a multiple of 4 or its
+// length is not a multiple of the stage is cut in up to three: a head of 1-3 steps (general
+// kernel) up to the next multiple of 4, the aligned middle (fast kernel), a tail of 1-7 steps
+// (general kernel).  The pieces run back to back on the stream; each starts from the state the
+// one before it stored.  *kernels receives the number of launches.
+cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s, VectorMapCache *cache, int *kernels)
+{
+    int launched = 1;
+    cudaError_t err;
+    const int head = (int)((4 - a.t0 % 4) % 4);
+    const int middle = a.T > head ? ((a.T - head) / kTmaStage) * kTmaStage : 0;
+    const uintptr_t bases = reinterpret_cast<uintptr_t>(a.obs) | reinterpret_cast<uintptr_t>(a.reward) |
+                            reinterpret_cast<uintptr_t>(a.done);
+    const bool cut = a.vector_path != kPathGeneral && a.frameskip == 1 && a.n % 16 == 0 && bases % 16 == 0 &&
+                     middle >= 2 * kTmaStage && middle != a.T;
+    if (!cut) {
+        err = launch_vector_one(a, s, cache);
+    } else {
+        launched = 0;
+        err = cudaSuccess;
+        const int tail = a.T - head - middle;
+        if (head > 0) {
+            err = launch_vector_one(sub_call(a, 0, head), s, nullptr);
+            ++launched;
+        }
+        if (err == cudaSuccess) {
+            err = launch_vector_one(sub_call(a, head, middle), s, cache);
+            ++launched;
+        }
+        if (err == cudaSuccess && tail > 0) {
+            err = launch_vector_one(sub_call(a, head + middle, tail), s, nullptr);
+            ++launched;
+        }
+    }
+    if (kernels != nullptr) *kernels = launched;
+    return err;
 }
 
 // ---- pixel rollout --------------------------------------------------------------------

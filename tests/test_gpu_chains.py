@@ -105,3 +105,32 @@ def test_every_path_gives_the_same_bytes_and_unaligned_calls_fall_through(torch_
         env = pong.PongEnv(16, 1)
         env.set_vector_path(7)
     assert e.value.code == -1
+
+
+@pytest.mark.parametrize("n,path", [(65536, pong.PATH_AUTO), (65536, pong.PATH_CHAINS), (4096, pong.PATH_AUTO),
+                                    (45056, pong.PATH_TMA)])
+def test_calls_that_start_or_end_off_the_grid_are_cut_and_still_match(torch_cuda, n, path):
+    """A call whose first step is no multiple of 4, or whose length is no multiple of 8, runs as a
+    short general-kernel head, a fast-kernel middle and a general-kernel tail (1 to 3 kernels):
+    the pieces must hand the state on exactly, in every action mode, and the kernel count shows
+    that the cut was taken."""
+    torch = torch_cuda
+    seed = 17
+    env = pong.PongEnv(n, seed, env_id_base=9)
+    env.set_vector_path(path)
+    ora = oracle.OraclePong(n, seed, env_id_base=9)
+    for k, (T, mode, kernels) in enumerate([(100, 0, 2), (1, 1, 1), (128, 1, 3), (37, 2, 3), (21, 3, 3), (23, 0, 3),
+                                            (128, 0, 3), (15, 0, 1), (3, 1, 1), (128, 0, 1)]):
+        before = env.launches
+        if mode == 2:
+            acts = explicit_actions(T, n, seed=k, repeat_fraction=0.3, odd_codes=True)
+            g, o = env.rollout(T, 2, torch.from_numpy(acts).cuda()), ora.rollout(T, 2, acts)
+        elif mode == 3:
+            g, o = env.rollout(T, 3, 1), ora.rollout(T, 3, 1)
+        else:
+            g, o = env.rollout(T, mode), ora.rollout(T, mode)
+        same(g, o, "cut call %d (T %d, mode %d)" % (k, T, mode))
+        assert env.launches - before == kernels, (k, T, env.launches - before)
+    assert env.get_state()[0].tobytes() == ora.get_state()[0].tobytes()
+    assert tuple(env.episode_stats()) == tuple(ora.episode_stats())
+    env.close()
