@@ -83,7 +83,7 @@ int do_rollout(pong_env *h, int T, int action_mode, const uint8_t *actions, int 
         err = pong::launch_rollout_vector(a, h->stream, &h->map_cache, &kernels);
     } else {
         a.ring = static_cast<uint8_t *>(obs);
-        err = pong::launch_rollout_pixels(a, h->sm_count, h->stream);
+        err = pong::launch_rollout_pixels(a, h->sm_count, h->stream, &kernels);
     }
     if (err != cudaSuccess) return PONG_ECUDA;
     h->launches += kernels;

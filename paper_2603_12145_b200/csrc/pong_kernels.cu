@@ -1013,7 +1013,7 @@ static int pixel_envs_per_block(int n, int sm_count, int max_per_block)
     }
 }
 
-cudaError_t launch_rollout_pixels(const LaunchArgs &a, int sm_count, cudaStream_t s)
+static cudaError_t launch_pixels_one(const LaunchArgs &a, int sm_count, cudaStream_t s)
 {
     cudaError_t err = cudaSuccess;
     if (a.t0 % 4 == 0 && a.T % 4 == 0) {
@@ -1052,6 +1052,40 @@ cudaError_t launch_rollout_pixels(const LaunchArgs &a, int sm_count, cudaStream_
     }
 #undef PONG_PIX
     return cudaGetLastError();
+}
+
+// A call that misses the four-steps-per-pass kernel only because it starts or ends off a
+// multiple of 4 is cut like a vector call: frame-at-a-time head (1-3 steps), four-step middle,
+// frame-at-a-time tail (16,384 envs x 64 steps from t = 1: 1412 us uncut).
+cudaError_t launch_rollout_pixels(const LaunchArgs &a, int sm_count, cudaStream_t s, int *kernels)
+{
+    int launched = 1;
+    cudaError_t err;
+    const int head = (int)((4 - a.t0 % 4) % 4);
+    const int middle = a.T > head ? ((a.T - head) / 4) * 4 : 0;
+    if (middle < 8 || middle == a.T) {
+        err = launch_pixels_one(a, sm_count, s);
+    } else {
+        launched = 0;
+        err = cudaSuccess;
+        const int tail = a.T - head - middle;
+        auto piece = [&](int from, int count) {
+            LaunchArgs b = a;
+            const size_t rows = (size_t)from * (size_t)a.n;
+            b.t0 = a.t0 + (unsigned long long)from;
+            b.T = count;
+            b.reward = a.reward + rows;
+            b.done = a.done + rows;
+            if (a.actions != nullptr && a.action_mode == 2) b.actions = a.actions + rows;
+            ++launched;
+            return launch_pixels_one(b, sm_count, s);
+        };
+        if (head > 0) err = piece(0, head);
+        if (err == cudaSuccess) err = piece(head, middle);
+        if (err == cudaSuccess && tail > 0) err = piece(head + middle, tail);
+    }
+    if (kernels != nullptr) *kernels = launched;
+    return err;
 }
 
 // One warp per env: paint the frame of the stored state and copy it to all

@@ -46,7 +46,7 @@ struct VectorMapCache {
 cudaError_t launch_reset(const LaunchArgs &a, cudaStream_t s);          // state + optional obs / ring
 cudaError_t launch_rollout_vector(const LaunchArgs &a, cudaStream_t s, VectorMapCache *cache = nullptr,
                                   int *kernels = nullptr);   // *kernels: how many kernels it launched (1-3)
-cudaError_t launch_rollout_pixels(const LaunchArgs &a, int sm_count, cudaStream_t s);
+cudaError_t launch_rollout_pixels(const LaunchArgs &a, int sm_count, cudaStream_t s, int *kernels = nullptr);
 cudaError_t launch_fill_actions(const LaunchArgs &a, int sticky, uint8_t *out, cudaStream_t s);
 cudaError_t launch_fill_words(const LaunchArgs &a, uint32_t *out, cudaStream_t s);
 cudaError_t launch_sample_actions(int n, const float *logits, const uint32_t *words, uint8_t *out,
